@@ -53,6 +53,7 @@ typedef enum {
 #define ZIPVL_DEV_BAD_INDEX 1u /* an entry of idx / probe_pos / seq_lens was out of range */
 #define ZIPVL_DEV_TIMEOUT 2u   /* a bounded wait inside a kernel ran out */
 #define ZIPVL_DEV_CAPACITY 4u  /* k or a cache length exceeded the capacity given */
+#define ZIPVL_DEV_BAD_VALUE 8u /* a score given to zipvl_select was negative or not a number */
 
 #define ZIPVL_BF16 0
 #define ZIPVL_F32 1
@@ -155,7 +156,9 @@ zipvl_status zipvl_score(const zipvl_layer *layer, const void *q, const void *k,
  * of its workspace.  mode: ZIPVL_BUDGET_BY_NORM, ZIPVL_TOPK_BY_ACC, ZIPVL_KEEP_LAST(r) or'ed
  * together; any other bit is ZIPVL_ERR_INVALID_ARG.
  *
- * acc, norm: device float[L] (non-negative).  k_out: device int32[1].
+ * acc, norm: device float[L], non-negative; a negative or NaN entry counts as zero in
+ * the sums, ranks by its bit pattern and is reported as ZIPVL_DEV_BAD_VALUE.
+ * k_out: device int32[1].
  * idx: device int32[L].  kept_mass: device float[1] or NULL.
  * ws: zipvl_workspace_bytes(ZIPVL_OP_SELECT).  L <= 2^20.
  */
@@ -181,6 +184,10 @@ zipvl_status zipvl_select(int32_t L, const float *acc, const float *norm, float 
  * between select and prefill; k_max: host upper bound on k used to size the
  * launch (pass L if unknown).  k > k_max is clamped and reported as
  * ZIPVL_DEV_CAPACITY.  out has the layer's dtype, contiguous.
+ * An entry of idx[0..k) outside [0, L) is reported as ZIPVL_DEV_BAD_INDEX: no memory
+ * is read or written for it (its output row is left alone, the rows of dropped
+ * tokens next to it are not cleared) and it stands in the attention of the later
+ * rows as an all-zero key and value.  k = 0 writes an all-zero PADDED output.
  */
 zipvl_status zipvl_sparse_prefill(const zipvl_layer *layer, const void *q, const void *k,
                                   const void *v, const int32_t *idx, const int32_t *k_dev,
@@ -238,7 +245,10 @@ zipvl_status zipvl_sparse_prefill_compact(const zipvl_layer *layer, const void *
  * device int32[B].  max_len: host upper bound on any seq_lens[b] after the
  * append; sizes the launch and the workspace.  A request whose cache is full
  * is not appended to and reports ZIPVL_DEV_CAPACITY; a request with zero rows
- * writes zeros.  The call enqueues two kernels (the second merges the cache chunks).
+ * writes zeros.  A request with seq_lens[b] < 0 or > capacity[b], or whose
+ * cache_off[b] is not a multiple of 16 bytes, is skipped as a whole (nothing of
+ * its cache is read or written, its output is zeros, its length stays) and
+ * reported as ZIPVL_DEV_BAD_INDEX.  The call enqueues two kernels (the second merges the cache chunks).
  */
 zipvl_status zipvl_decode(const zipvl_decode_desc *desc, const void *q, const void *k_new,
                           const void *v_new, void *k_cache, void *v_cache,
@@ -268,8 +278,10 @@ zipvl_status zipvl_decode(const zipvl_decode_desc *desc, const void *q, const vo
  * workspace.
  *
  * The first call on each device looks up the array's device address (with that
- * device current) and caches it; make that first call before starting any
- * stream capture.  All calls share the one array and it keeps the previous
+ * device current) and caches it for the life of the process; make that first
+ * call before starting any stream capture.  The cached address belongs to the
+ * device's primary context: after cudaDeviceReset it is stale and this entry
+ * point must not be used again in the process.  All calls share the one array and it keeps the previous
  * call's contents: nothing in it has to start at zero, every slot a call reads
  * was written by that same call.  Two calls that overlap on the GPU
  * (different streams, no ordering between them) race on it: order them.
@@ -304,6 +316,21 @@ zipvl_status zipvl_prefill_layer_host(const zipvl_layer *layer, const void *q, c
  * zipvl_prefill_layer_host never ran on the device.
  */
 zipvl_status zipvl_release_host_scratch(void);
+
+/*
+ * zipvl_selftest_wait_timeout -- run a bounded device wait out, on purpose and harmlessly.
+ * (No counterpart in the paper: a check of the library's own failure handling.)
+ * Every wait inside the tensor-core kernels gives up after a fixed number of polls, raises
+ * its thread block's abort flag, lets all warps leave through the common exit and reports
+ * ZIPVL_DEV_TIMEOUT.  This call launches one 128-thread block that uses that same wait:
+ * warp 0 waits on a barrier that completes, warps 1-3 on one that nobody arrives at, each
+ * for at most poll_limit polls (1 .. 2^20).  The kernel always returns; afterwards
+ * status_word has ZIPVL_DEV_TIMEOUT set and progress[0..4) (device int32, may be NULL)
+ * holds 1 for the warp whose wait succeeded and 0 for the three that gave up.  The CUDA
+ * context stays usable.
+ */
+zipvl_status zipvl_selftest_wait_timeout(int32_t poll_limit, int32_t *progress,
+                                         int32_t *status_word, void *stream);
 
 #ifdef __cplusplus
 }

@@ -19,14 +19,14 @@ ZIPVL_BF16, ZIPVL_F32, ZIPVL_F16 = 0, 1, 2
 OP_SCORE, OP_SELECT, OP_SPARSE_PREFILL, OP_COMPACT_KV, OP_DECODE = range(5)
 BUDGET_BY_NORM, TOPK_BY_ACC = 1, 2
 OUT_PADDED, OUT_COMPACT = 0, 1
-DEV_BAD_INDEX, DEV_TIMEOUT, DEV_CAPACITY = 1, 2, 4
+DEV_BAD_INDEX, DEV_TIMEOUT, DEV_CAPACITY, DEV_BAD_VALUE = 1, 2, 4, 8
 
 EXPORTS = ["zipvl_status_string", "zipvl_last_error", "zipvl_version", "zipvl_launch_count",
            "zipvl_workspace_bytes",
            "zipvl_score", "zipvl_select", "zipvl_sparse_prefill", "zipvl_compact_kv",
            "zipvl_sparse_prefill_compact",
            "zipvl_decode", "zipvl_decode_noalloc", "zipvl_prefill_layer_host",
-           "zipvl_release_host_scratch"]
+           "zipvl_release_host_scratch", "zipvl_selftest_wait_timeout"]
 
 
 class ZipvlError(RuntimeError):
@@ -89,6 +89,8 @@ def load():
                                          vp, i32, vp, vp, vp]
     lib.zipvl_prefill_layer_host.restype = C.c_int
     lib.zipvl_prefill_layer_host.argtypes = [lp, vp, vp, vp, vp, i32, f32, vp, vp, vp, vp, vp]
+    lib.zipvl_selftest_wait_timeout.restype = C.c_int
+    lib.zipvl_selftest_wait_timeout.argtypes = [i32, vp, vp, vp]
     _lib = lib
     return lib
 
@@ -282,6 +284,13 @@ def zipvl_decode_noalloc(desc, q, k_new, v_new, k_cache, v_cache, cache_off, cap
                                        _ptr(capacity), _ptr(seq_lens), int(max_len), _ptr(out),
                                        _ptr(status), _stream(stream)))
     return out
+
+
+def zipvl_selftest_wait_timeout(poll_limit, progress, status, stream=None):
+    """Launch the library's bounded-wait self-test (see include/zipvl.h)."""
+    _dev(progress, "progress", torch.int32), _dev(status, "status", torch.int32)
+    _check(load().zipvl_selftest_wait_timeout(int(poll_limit), _ptr(progress), _ptr(status),
+                                              _stream(stream)))
 
 
 def zipvl_prefill_layer_host(layer, q, k, v, probe_pos, tau, out=None, k_cache=None, v_cache=None,

@@ -2,6 +2,7 @@
 // No kernel lives here.  Every entry point validates on the host, launches on
 // the caller's stream and returns without synchronising.
 #include <math.h>
+#include <mutex>
 #include <stdarg.h>
 #include <stdio.h>
 #include <string.h>
@@ -269,12 +270,14 @@ namespace {
 // call on a 2944-token layer).  zipvl_release_host_scratch() gives the memory back.
 constexpr int kMaxDevices = 64;
 cudaMemPool_t g_host_pool[kMaxDevices] = {};
+std::mutex g_host_pool_mutex;   // two first calls on one device must not both create a pool
 
 cudaError_t host_pool(cudaMemPool_t *pool) {
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_host_pool_mutex);
     if (!g_host_pool[dev]) {
         cudaMemPoolProps props = {};
         props.allocType = cudaMemAllocationTypePinned;
@@ -298,6 +301,7 @@ zipvl_status zipvl_release_host_scratch(void) {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices)
         return fail(ZIPVL_ERR_CUDA, "zipvl_release_host_scratch: no current device");
+    std::lock_guard<std::mutex> lock(g_host_pool_mutex);
     if (g_host_pool[dev]) {
         const cudaError_t e = cudaMemPoolTrimTo(g_host_pool[dev], 0);
         if (e != cudaSuccess)

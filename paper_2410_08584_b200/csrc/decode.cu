@@ -80,10 +80,17 @@ decode_kernel(int Hq, int Hkv, float scale_log2, const T *__restrict__ q,
     const bool first = blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0;
 
     // Eq. 4: the new row goes to position seq_lens[b] if the cache has room
+    // A request whose length is negative or beyond its capacity, or whose cache offset breaks
+    // the 16-byte alignment of the row loads, is skipped as a whole (no load, no append, a
+    // zero output) and reported: none of its rows can be trusted to lie inside the cache.
     const int old_len = seq_lens[b];
-    const bool appended = k_new != nullptr && old_len >= 0 && old_len < capacity[b];
-    if (k_new != nullptr && !appended && first) report(status_word, ZIPVL_DEV_CAPACITY);
-    int len = max(old_len, 0) + (appended ? 1 : 0);
+    const int cap = capacity[b];
+    const bool bad = old_len < 0 || old_len > cap ||
+                     ((cache_off[b] * (long long)sizeof(T)) & 15) != 0;
+    if (bad && first) report(status_word, ZIPVL_DEV_BAD_INDEX);
+    const bool appended = !bad && k_new != nullptr && old_len < cap;
+    if (k_new != nullptr && !bad && !appended && first) report(status_word, ZIPVL_DEV_CAPACITY);
+    int len = bad ? 0 : old_len + (appended ? 1 : 0);
     if (len > max_len) {
         if (first) report(status_word, ZIPVL_DEV_CAPACITY);
         len = max_len;
@@ -345,8 +352,8 @@ zipvl_status launch_decode(const zipvl_decode_desc &d, float scale_log2, const v
 
 // ---- decode without any allocation ------------------------------------------
 // Scratch for zipvl_decode_noalloc: the per-chunk (m, l, o) partials and the
-// tickets live in this file-scope device array instead of a caller-supplied
-// workspace.  Every GPU that loads the library holds these 8 MiB until the
+// per-request (length, appended) pairs live in this file-scope device array
+// instead of a caller-supplied workspace.  Every GPU that loads the library holds these 8 MiB until the
 // process exits.
 constexpr size_t kNoAllocScratchBytes = 8u << 20;
 static __device__ __align__(256) unsigned char g_decode_scratch[kNoAllocScratchBytes];

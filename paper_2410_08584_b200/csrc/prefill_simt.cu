@@ -38,6 +38,11 @@ prefill_simt_kernel(LayerArgs a, const T *__restrict__ q, const T *__restrict__ 
     }
     const int h = blockIdx.y, g = h / a.G;
     const int i0 = blockIdx.x * kBM;
+    if (n == 0 && blockIdx.x == 0 && out_mode == ZIPVL_OUT_PADDED) {
+        // nothing kept: every row is a dropped token's row
+        for (long long e = threadIdx.x; e < (long long)a.L * D; e += kPfThreads)
+            store_elem(out + ((e / D) * a.Hq + h) * D + (e % D), 0.f);
+    }
     if (i0 >= n) return;
     const int i1 = min(n, i0 + kBM);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -47,7 +52,7 @@ prefill_simt_kernel(LayerArgs a, const T *__restrict__ q, const T *__restrict__ 
         const int row = e / (D / 8), col = (e % (D / 8)) * 8;
         float x[8];
         int t = (i0 + row < i1) ? idx[i0 + row] : -1;
-        if (t >= a.L) { report(status_word, ZIPVL_DEV_BAD_INDEX); t = -1; }
+        if (i0 + row < i1 && (t < 0 || t >= a.L)) { report(status_word, ZIPVL_DEV_BAD_INDEX); t = -1; }
         if (t >= 0) {
             load8(q + (long long)t * a.q_stride + (long long)h * D + col, x);
         } else {
@@ -74,7 +79,7 @@ prefill_simt_kernel(LayerArgs a, const T *__restrict__ q, const T *__restrict__ 
             const int row = e / (D / 8), col = (e % (D / 8)) * 8;
             float x[8], y[8];
             int t = (jt + row < i1) ? idx[jt + row] : -1;
-            if (t >= a.L) t = -1;
+            if (t < 0 || t >= a.L) t = -1;
             if (t >= 0) {
                 const long long off = (long long)t * a.kv_stride + (long long)g * D + col;
                 load8(k + off, x);
@@ -157,7 +162,13 @@ prefill_simt_kernel(LayerArgs a, const T *__restrict__ q, const T *__restrict__ 
 #pragma unroll
         for (int c = 0; c < CPL; ++c) store_elem(dst + lane + 32 * c, o[r][c] * inv);
         if (out_mode == ZIPVL_OUT_PADDED) {
-            const int lo = (i == 0) ? 0 : idx[i - 1] + 1;
+            // the gap in front of this token; a previous entry that is out of range or not
+            // below this one (the list must ascend) is read as "no gap"
+            int lo = 0;
+            if (i > 0) {
+                const int tp = idx[i - 1];
+                lo = (tp >= 0 && tp < t) ? tp + 1 : t;
+            }
             for (int z = lo; z < t; ++z) {
                 T *zr = out + ((long long)z * a.Hq + h) * D;
 #pragma unroll

@@ -164,8 +164,9 @@ prefill_tc_kernel(LayerArgs a, const __nv_bfloat16 *__restrict__ q,
     // barrier, so its latency hides behind it: a softmax thread's own query row, a
     // producer lane's row of key tile 0.
     auto token_of = [&](int i) {
-        int t = (i < n_valid) ? idx[i] : -1;
-        if (t >= a.L) { report(status_word, ZIPVL_DEV_BAD_INDEX); t = -1; }
+        if (i >= n_valid) return -1;
+        int t = idx[i];
+        if (t < 0 || t >= a.L) { report(status_word, ZIPVL_DEV_BAD_INDEX); t = -1; }
         return t;
     };
     int first_tok = -1;
@@ -179,6 +180,16 @@ prefill_tc_kernel(LayerArgs a, const __nv_bfloat16 *__restrict__ q,
     const uint32_t tmem = bar->tmem_base;
     if (no_work) {                                  // a CTA past the kept set: give the columns back
         if (warp == 12) tmem_dealloc(tmem, kTmemCols);
+        if (n_valid == 0 && blockIdx.y == 0 && (int)blockIdx.x < a.Hq) {
+            // nothing kept: the results are those of the two separate calls -- an all-zero
+            // PADDED output (every row is a dropped token's) and a cache of length 0
+            if (out_mode == ZIPVL_OUT_PADDED) {
+                const uint4 z = make_uint4(0, 0, 0, 0);
+                for (int e = threadIdx.x; e < a.L * 16; e += kThreadsTc)
+                    reinterpret_cast<uint4 *>(out + ((long long)(e >> 4) * a.Hq + h) * kD)[e & 15] = z;
+            }
+            if (kc != nullptr && blockIdx.x == 0 && threadIdx.x == 0) *len_out = 0;
+        }
         return;
     }
 
@@ -238,8 +249,10 @@ prefill_tc_kernel(LayerArgs a, const __nv_bfloat16 *__restrict__ q,
                     const int t = token_of(i);
                     int lo = 0, hi = 0;                       // my gap: rows [lo, hi)
                     if (t >= 0) {
+                        // a previous entry that is out of range, or not below this one (the
+                        // list must ascend), is read as "no gap": nothing is cleared for it
                         const int tp = (i == 0) ? -1 : idx[i - 1];
-                        lo = (tp >= a.L) ? t : tp + 1;        // (a bad previous index: no gap)
+                        lo = (i == 0) ? 0 : ((tp >= 0 && tp < t) ? tp + 1 : t);
                         hi = t;
                     }
                     const bool last = (t >= 0 && i == n_valid - 1);

@@ -415,7 +415,7 @@ template <bool kKeepLast>   // (the option outside the paper is its own instanti
 __global__ void __launch_bounds__(kSelThreads)
 select_kernel(int L, const float *__restrict__ acc, const float *__restrict__ norm, float tau,
               uint32_t mode, int fixed_k, int32_t *__restrict__ k_out, int32_t *__restrict__ idx,
-              float *__restrict__ kept_mass, GlobalHist *__restrict__ gh) {
+              float *__restrict__ kept_mass, GlobalHist *__restrict__ gh, int32_t *status_word) {
     extern __shared__ __align__(16) unsigned char sel_dyn[];
     SelSmem &sm = *reinterpret_cast<SelSmem *>(sel_dyn);
     __shared__ SelCtl c;
@@ -434,6 +434,7 @@ select_kernel(int L, const float *__restrict__ acc, const float *__restrict__ no
     // shared memory; several CTAs take 1024 tokens each and meet in the global one
     const bool solo = (gridDim.x == 1);
     unsigned long long my_sum = 0;                 // this thread's share of S (used when solo)
+    bool bad_value = false;                        // a score that is negative or not a number
     const int row_end = solo ? L : min(L, (int)(blockIdx.x + 1) * kSelThreads);
     for (int jb = blockIdx.x * kSelThreads; jb < row_end; jb += kSelThreads * kBatch) {
         float vbs[kBatch], vrs[kBatch];            // the loads of a batch are in flight together
@@ -449,10 +450,14 @@ select_kernel(int L, const float *__restrict__ acc, const float *__restrict__ no
             const bool act = jb + u * kSelThreads + (int)threadIdx.x < row_end;
             const unsigned long long fxb = act ? to_fx(vbs[u]) : 0ull;
             my_sum += fxb;
+            bad_value |= act && (!(vbs[u] >= 0.f) || !(vrs[u] >= 0.f));
             hist_add(sm.cnt_b, &sm, act, float_key(vbs[u]) >> 20, fxb, &c.rng[0]);
             hist_add(sm.cnt_r, nullptr, act, float_key(vrs[u]) >> 20, 0ull, &c.rng[2]);
         }
     }
+    // (such a score counts as zero in the sums and ranks by its bit pattern; the call
+    // still completes, the caller is told)
+    if (bad_value) report(status_word, ZIPVL_DEV_BAD_VALUE);
     __syncthreads();
     if (!solo) {
     for (int b = threadIdx.x; b < kBins; b += kSelThreads) {
@@ -614,7 +619,6 @@ size_t select_ws_bytes() { return (sizeof(GlobalHist) + 255) & ~(size_t)255; }
 zipvl_status launch_select(int L, const float *acc, const float *norm, float tau, uint32_t mode,
                            int fixed_k, int32_t *k_out, int32_t *idx, float *kept_mass, void *ws,
                            int32_t *status_word, cudaStream_t st) {
-    (void)status_word;
     auto kernel = (mode >> 8) ? select_kernel<true> : select_kernel<false>;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)sizeof(SelSmem));
@@ -622,7 +626,7 @@ zipvl_status launch_select(int L, const float *acc, const float *norm, float tau
     if (e == cudaSuccess && grid > 1) e = cudaMemsetAsync(ws, 0, sizeof(GlobalHist), st);
     if (e != cudaSuccess) return fail(ZIPVL_ERR_CUDA, "select: %s", cudaGetErrorString(e));
     e = launch_dependent(kernel, dim3(grid), dim3(kSelThreads), sizeof(SelSmem), st, L, acc, norm, tau,
-                         mode, fixed_k, k_out, idx, kept_mass, reinterpret_cast<GlobalHist *>(ws));
+                         mode, fixed_k, k_out, idx, kept_mass, reinterpret_cast<GlobalHist *>(ws), status_word);
     if (e != cudaSuccess) return fail(ZIPVL_ERR_CUDA, "select: launch: %s", cudaGetErrorString(e));
     count_launches(1);
     return check_launch("zipvl_select");

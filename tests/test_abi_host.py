@@ -109,6 +109,18 @@ def test_argument_validation_without_a_device(lib):
     assert lib.zipvl_decode(C.byref(d), p, p, p, p, p, p, p, p, 10, p, p, 8, None, None) == 3
     d9 = z.zipvl_decode_desc(2, 18, 2, 64, 0, 0.0)
     assert lib.zipvl_decode(C.byref(d9), p, p, p, p, p, p, p, p, 10, p, p, 1 << 20, None, None) == 2
+    # decode without a workspace: the same validation, and the size check of its built-in
+    # scratch, before anything is launched
+    na = lib.zipvl_decode_noalloc
+    assert na(C.byref(d), null, None, None, p, p, p, p, p, 128, p, None, None) == 1
+    assert na(C.byref(d), p, p, null, p, p, p, p, p, 128, p, None, None) == 1
+    big = z.zipvl_decode_desc(16, 32, 32, 128, 0, 0.0)
+    rc, text = status(lambda: na(C.byref(big), p, None, None, p, p, p, p, p, 32768, p, None, None))
+    assert rc == 3 and "scratch" in text
+    # the wait self-test: limits outside [1, 2^20] and a missing status word are refused
+    assert lib.zipvl_selftest_wait_timeout(0, None, p, None) == 1
+    assert lib.zipvl_selftest_wait_timeout(1 << 21, None, p, None) == 1
+    assert lib.zipvl_selftest_wait_timeout(1000, None, None, None) == 1
     assert lib.zipvl_status_string(3).decode() == "workspace too small"
     assert lib.zipvl_status_string(0).decode() == "ok"
 

@@ -393,6 +393,208 @@ def test_bad_index_is_reported_not_fatal(zipvl):
     assert n.item() == 50 and st.item() & zipvl.DEV_CAPACITY
 
 
+@pytest.mark.parametrize("name", ["ragged_129", "tiny_fp32_d128"])     # tensor-core and CUDA-core kernels
+def test_negative_index_is_skipped_and_writes_nothing_out_of_bounds(zipvl, name):
+    """A negative entry inside [0, k): reported, its row skipped, no store in front of `out`
+    (canary rows on both sides stay untouched) and every other row as in the clean run."""
+    layer = CASES[name]()
+    q, k, v, probe = put(layer)
+    L, Hq, d = layer.L, layer.n_q_heads, layer.head_dim
+    desc = zipvl.layer_desc(q, k)
+    idx = torch.arange(L, dtype=torch.int32, device=DEV)
+    k_dev = torch.tensor([L], dtype=torch.int32, device=DEV)
+    st = status_word()
+    clean = zipvl.zipvl_sparse_prefill(desc, q, k, v, idx, k_dev, L, status=st)
+    torch.cuda.synchronize()
+    assert st.item() == 0
+    canary = 77.0
+    guard = 16                                          # rows in front of and behind the output
+    buf = torch.full((L + 2 * guard, Hq, d), canary, dtype=q.dtype, device=DEV)
+    out = buf[guard:guard + L]
+    bad = idx.clone()
+    bad[3] = -7
+    zipvl.zipvl_sparse_prefill(desc, q, k, v, bad, k_dev, L, out=out, status=st)
+    torch.cuda.synchronize()
+    assert st.item() & zipvl.DEV_BAD_INDEX
+    assert torch.all(buf[:guard] == canary) and torch.all(buf[guard + L:] == canary)
+    # rows 0..2 do not see entry 3 at all: the bits of the clean run.  The bad entry's own
+    # row is not written; the later rows saw an all-zero key and value in its place (the
+    # documented stand-in), so they are finite and close to, not equal to, the clean run.
+    assert torch.equal(out[:3], clean[:3])
+    assert torch.all(out[3] == canary)
+    assert torch.isfinite(out[4:].float()).all()
+    # the fused call and the compaction see the same list
+    st.zero_()
+    kc, vc = torch.zeros_like(k), torch.zeros_like(v)
+    buf.fill_(canary)
+    zipvl.zipvl_sparse_prefill_compact(desc, q, k, v, bad, k_dev, L, kc, vc, L, out=out, status=st)
+    torch.cuda.synchronize()
+    assert st.item() & zipvl.DEV_BAD_INDEX
+    assert torch.all(buf[:guard] == canary) and torch.all(buf[guard + L:] == canary)
+    assert torch.equal(kc[4:], k[4:]) and torch.equal(kc[:3], k[:3])
+
+
+@pytest.mark.parametrize("name", ["ragged_129", "tiny_fp32_d128"])
+def test_empty_selection_zeroes_the_output_and_the_cache_length(zipvl, name):
+    """k = 0 on the device: the padded output is all zeros, the cache length is 0, for the
+    separate calls and for the fused one alike."""
+    layer = CASES[name]()
+    q, k, v, probe = put(layer)
+    L = layer.L
+    desc = zipvl.layer_desc(q, k)
+    idx = torch.full((L,), -1, dtype=torch.int32, device=DEV)
+    k_dev = torch.zeros(1, dtype=torch.int32, device=DEV)
+    st = status_word()
+    out = torch.full_like(q, 5.0)
+    zipvl.zipvl_sparse_prefill(desc, q, k, v, idx, k_dev, L, out=out, status=st)
+    kc, vc = torch.zeros_like(k), torch.zeros_like(v)
+    n = zipvl.zipvl_compact_kv(desc, k, v, idx, k_dev, L, kc, vc, L, status=st)
+    out2 = torch.full_like(q, 5.0)
+    n2 = torch.full((1,), 99, dtype=torch.int32, device=DEV)
+    zipvl.zipvl_sparse_prefill_compact(desc, q, k, v, idx, k_dev, L, kc, vc, L, out=out2, len_out=n2, status=st)
+    torch.cuda.synchronize()
+    assert st.item() == 0
+    assert not out.any() and not out2.any()
+    assert n.item() == 0 and n2.item() == 0
+
+
+def test_select_reports_negative_and_nan_scores(zipvl):
+    g = torch.Generator().manual_seed(3)
+    acc = torch.rand(500, generator=g).to(DEV)
+    norm = torch.rand(500, generator=g).to(DEV)
+    st = status_word()
+    zipvl.zipvl_select(acc, norm, 0.9, status=st)
+    torch.cuda.synchronize()
+    assert st.item() == 0
+    for bad_val, which in ((-1.0, 0), (float("nan"), 1)):
+        a, n = acc.clone(), norm.clone()
+        (a if which == 0 else n)[17] = bad_val
+        st.zero_()
+        k_dev, idx = zipvl.zipvl_select(a, n, 0.9, status=st)
+        torch.cuda.synchronize()
+        assert st.item() & zipvl.DEV_BAD_VALUE
+        kk = int(k_dev.item())
+        assert 1 <= kk <= 500 and idx[:kk].min().item() >= 0       # the call still completes
+
+
+def test_a_bounded_wait_that_runs_out_is_reported_and_the_context_survives(zipvl):
+    """The wait every tensor-core kernel uses, on a barrier nobody arrives at, with a poll
+    limit of a few thousand: the kernel returns, ZIPVL_DEV_TIMEOUT is set, the warp whose
+    barrier did complete is unaffected, and the next parity call runs as usual."""
+    st = status_word()
+    progress = torch.full((4,), -1, dtype=torch.int32, device=DEV)
+    zipvl.zipvl_selftest_wait_timeout(4000, progress, st)
+    torch.cuda.synchronize()
+    assert st.item() == zipvl.DEV_TIMEOUT
+    assert progress.tolist() == [1, 0, 0, 0]
+    layer = CASES["ragged_129"]()
+    r = gpu_pipeline(zipvl, layer)
+    assert r["status"] == 0 and r["k"] >= 1
+
+
+def test_decode_skips_requests_with_impossible_lengths_or_offsets(zipvl):
+    """seq_lens < 0, seq_lens > capacity and a cache offset off the 16-byte grid: the request
+    is skipped (zero output, cache and length untouched) and reported; the other requests of
+    the batch are served as usual.  All buffers are in range, so nothing can fault."""
+    lens, Hq, Hkv, d = [40, 300, 77, 130], 4, 2, 128
+    B = len(lens)
+    kc, vc, off, cap = build_caches(lens, Hkv, d, torch.bfloat16, 4, seed=8)
+    g = torch.Generator().manual_seed(9)
+    q = torch.randn(B, Hq, d, generator=g).bfloat16()
+    kn = torch.randn(B, Hkv, d, generator=g).bfloat16()
+    vn = torch.randn(B, Hkv, d, generator=g).bfloat16()
+    desc = zipvl.zipvl_decode_desc(B, Hq, Hkv, d, zipvl.ZIPVL_BF16, 0.0)
+    seq_bad = torch.tensor([-3, 300, 77 + 50, 130], dtype=torch.int32)     # request 0 and 2 impossible
+    off_bad = off.clone()
+    off_bad[3] += 4                                                         # request 3: 8 bytes off
+    kc_d, vc_d = kc.to(DEV), vc.to(DEV)
+    seq_d = seq_bad.to(DEV)
+    st = status_word()
+    out = zipvl.zipvl_decode(desc, q.to(DEV), kn.to(DEV), vn.to(DEV), kc_d, vc_d, off_bad.to(DEV),
+                             cap.to(DEV), seq_d, max(lens) + 4, status=st)
+    torch.cuda.synchronize()
+    assert st.item() & zipvl.DEV_BAD_INDEX
+    assert seq_d.tolist() == [-3, 301, 127, 130]
+    assert not out[0].any() and not out[2].any() and not out[3].any()
+    # request 1 is the oracle's answer
+    ko, vo = to_np(kc).copy(), to_np(vc).copy()
+    seqo = np.array(lens, np.int32)
+    ref = oracle.decode_step(to_np(q), to_np(kn), to_np(vn), ko, vo, off.numpy(), seqo, Hkv)
+    check_attention(to_np(out)[1], ref[1], torch.bfloat16)
+    # and only request 1's cache row changed
+    kc_after = kc_d.cpu()
+    row = Hkv * d
+    o1 = int(off[1]) + 300 * row
+    assert torch.equal(kc_after[o1:o1 + row], kn[1].reshape(-1))
+    kc_after[o1:o1 + row] = kc[o1:o1 + row]
+    assert torch.equal(kc_after, kc)
+
+
+def test_all_rows_as_probes_on_16_bit_inputs(zipvl):
+    """More probe rows than one tensor-core tile holds (the "all tokens" probe strategy of the
+    supplementary ablation at L = 300): exact full-attention column sums on bf16 inputs."""
+    layer = W.heavy_key_layer(L_visual=260, L_text=40, H=4, seed=41)
+    layer.probe_pos = torch.arange(layer.L, dtype=torch.int32)
+    r = gpu_pipeline(zipvl, layer)
+    assert r["status"] == 0
+    qf, kf = to_np(layer.q), to_np(layer.k)
+    acc_ref, S = oracle.probe_scores(qf, kf, layer.probe_pos.numpy())
+    norm_ref, nnz = oracle.normalise(acc_ref, layer.probe_pos.numpy(), layer.n_q_heads)
+    assert np.array_equal(nnz, layer.L - np.arange(layer.L))
+    check_scores(r["acc"], r["norm"], acc_ref, norm_ref, S)
+    check_select(r["k"], r["idx"], r["acc"].astype(np.float64), r["norm"].astype(np.float64), layer.tau)
+
+
+def _tiny_shape_case(zipvl, L, H, G, d, n_probe, tau, dtype, seed):
+    Hkv = H
+    Hq = H * G
+    g = torch.Generator().manual_seed(seed)
+    q = torch.randn(L, Hq, d, generator=g).to(dtype)
+    k = (torch.randn(L, Hkv, d, generator=g) * (1.0 + 2.0 * (torch.rand(L, 1, 1, generator=g) < 0.2))).to(dtype)
+    v = torch.randn(L, Hkv, d, generator=g).to(dtype)
+    P = min(n_probe, L)
+    # P distinct rows, ascending, the last row always among them
+    probe = torch.unique(torch.cat([torch.randperm(L, generator=g)[:P - 1],
+                                    torch.tensor([L - 1])])).to(torch.int32)
+    layer = W.Layer("tiny_shape", q, k, v, probe, tau)
+    r = gpu_pipeline(zipvl, layer)
+    assert r["status"] == 0
+    qf, kf, vf = to_np(q), to_np(k), to_np(v)
+    acc_ref, S = oracle.probe_scores(qf, kf, probe.numpy())
+    norm_ref, _ = oracle.normalise(acc_ref, probe.numpy(), Hq)
+    err = check_scores(r["acc"], r["norm"], acc_ref, norm_ref, S)
+    check_select(r["k"], r["idx"], r["acc"].astype(np.float64), r["norm"].astype(np.float64), tau)
+    check_select(r["k"], r["idx"], acc_ref, norm_ref, tau, eps=max(1e-6, 4 * err))
+    T = r["idx"][: r["k"]]
+    ref = oracle.sparse_prefill(qf, kf, vf, T)
+    out = to_np(r["out"])
+    check_attention(out[T], ref, dtype)
+    assert not out[np.setdiff1d(np.arange(L), T)].any()
+    Tl = torch.from_numpy(T.astype(np.int64))
+    assert r["len"] == r["k"] and torch.equal(r["kc"][: r["k"]].cpu(), k[Tl]) and torch.equal(r["vc"][: r["k"]].cpu(), v[Tl])
+
+
+def test_generated_tiny_shapes(zipvl):
+    """Property-style sweep over small shapes drawn by hypothesis (fixed seed): odd lengths,
+    one token, more probes than tokens, one probe, grouped heads, every storage type, budgets
+    from one token to everything -- the whole chain against the oracle."""
+    from hypothesis import HealthCheck, given, seed, settings
+    from hypothesis import strategies as hs
+
+    @seed(20241008)
+    @settings(max_examples=40, deadline=None, derandomize=True,
+              suppress_health_check=list(HealthCheck))
+    @given(L=hs.integers(1, 300), H=hs.integers(1, 3), G=hs.sampled_from([1, 2, 7]),
+           d=hs.sampled_from([64, 128]), n_probe=hs.sampled_from([1, 5, 64, 128, 400]),
+           tau=hs.sampled_from([0.3, 0.9, 0.97, 1.0]),
+           dtype=hs.sampled_from([torch.bfloat16, torch.float16, torch.float32]),
+           s=hs.integers(0, 10 ** 6))
+    def run(L, H, G, d, n_probe, tau, dtype, s):
+        _tiny_shape_case(zipvl, L, H, G, d, n_probe, tau, dtype, s)
+
+    run()
+
+
 # ----------------------------------------------------------------------------
 # decode (Algorithm 2)
 # ----------------------------------------------------------------------------
