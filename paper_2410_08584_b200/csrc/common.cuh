@@ -79,7 +79,20 @@ __device__ __forceinline__ uint32_t float_key(float v) {
 // touches global memory only behind grid_dependency_wait(), which returns when every
 // earlier kernel in the stream has completed and its writes are visible.  Next to a
 // kernel launched without the attribute both instructions do nothing.
-__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+//
+// The pointers through which the kernel then reads what an earlier kernel wrote are handed
+// to the wait and come back "redefined" by an empty asm statement.  Without that, a load
+// through a `const T *__restrict__` parameter -- or through any restrict parameter the
+// kernel never stores to -- counts as a load of invariant memory, which the compiler may
+// schedule above every barrier, the wait included: a decode step replayed from a CUDA
+// graph read the cache length of the replay before, because that one load had moved up.
+template <typename T>
+__device__ __forceinline__ void redefine_pointer(T &p) { asm volatile("" : "+l"(p)::"memory"); }
+template <typename... P>
+__device__ __forceinline__ void grid_dependency_wait(P &...ptrs) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    (redefine_pointer(ptrs), ...);
+}
 __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 template <typename... KArgs, typename... Args>

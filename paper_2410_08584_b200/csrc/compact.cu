@@ -20,7 +20,7 @@ compact_kernel(const uint4 *__restrict__ k, const uint4 *__restrict__ v,
                uint4 *__restrict__ vc, int capacity, int32_t *__restrict__ len_out,
                int32_t *status_word) {
     grid_launch_dependents();
-    grid_dependency_wait();       // k_dev and idx are the previous kernel's output
+    grid_dependency_wait(k, v, idx, k_dev);   // k_dev and idx are the previous kernel's output
     int n = *k_dev;
     const int lim = min(k_max, capacity);
     if (n > lim || n < 0) {

@@ -70,7 +70,8 @@ decode_kernel(int Hq, int Hkv, float scale_log2, const T *__restrict__ q,
     __shared__ float sm_m[NG][GT], sm_l[NG][GT];
 
     grid_launch_dependents();
-    grid_dependency_wait();       // lengths and caches may be the previous kernel's output
+    // lengths and caches may be the previous kernel's output
+    grid_dependency_wait(q, k_new, v_new, k_cache, v_cache, cache_off, capacity, seq_lens);
     const int G = Hq / Hkv;
     const int q_tiles = (G + GT - 1) / GT;
     const int hkv = blockIdx.y / q_tiles, qt = blockIdx.y % q_tiles;
@@ -237,7 +238,7 @@ __global__ void __launch_bounds__(256)
 decode_merge_kernel(int Hq, int chunk, int n_chunks, const float *__restrict__ ws,
                     const int *__restrict__ lens, int32_t *__restrict__ seq_lens, T *__restrict__ out) {
     grid_launch_dependents();
-    grid_dependency_wait();
+    grid_dependency_wait(ws, lens, seq_lens);
     const int b = blockIdx.y;
     const int len = lens[2 * b];
     const int n_valid_chunks = (len + chunk - 1) / chunk;

@@ -140,7 +140,7 @@ prefill_tc_kernel(LayerArgs a, const __nv_bfloat16 *__restrict__ q,
         fence_barrier_init();
     }
     if (warp == 12) tmem_alloc(smem_u32(&bar->tmem_base), kTmemCols);
-    grid_dependency_wait();       // k_dev and idx are the previous kernel's output
+    grid_dependency_wait(q, k, v, idx, k_dev);   // k_dev and idx are the previous kernel's output
     int n_valid = *k_dev;
     if (n_valid > k_max || n_valid < 0) {
         if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0)

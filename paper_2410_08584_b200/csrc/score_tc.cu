@@ -103,7 +103,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap kmap, LayerArgs a,
     // <0> may have been staged behind the caller's previous kernel: no global access before
     // that kernel is complete.  <1> only follows <0>, which triggers it at its very end, so
     // the inputs are settled; it waits further down, just before it reads <0>'s results.
-    if (MODE == 0) grid_dependency_wait();
+    if (MODE == 0) grid_dependency_wait(q, probe_pos);
     else grid_launch_dependents();
     // probe positions
     if (threadIdx.x < kMaxProbe) {
@@ -184,7 +184,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap kmap, LayerArgs a,
             // Everything above (and the K loads and the first QK of the other warps) may
             // run while the statistics kernel is still finishing; its results are read
             // only behind this point.
-            grid_dependency_wait();
+            grid_dependency_wait(stats);
             const int r = row, c = sPos[row];
             float M = -INFINITY, Ls = 0.f;
             if (c >= 0) {

@@ -419,8 +419,6 @@ select_kernel(int L, const float *__restrict__ acc, const float *__restrict__ no
     extern __shared__ __align__(16) unsigned char sel_dyn[];
     SelSmem &sm = *reinterpret_cast<SelSmem *>(sel_dyn);
     __shared__ SelCtl c;
-    const float *bud = (mode & ZIPVL_BUDGET_BY_NORM) ? norm : acc;
-    const float *rank = (mode & ZIPVL_TOPK_BY_ACC) ? acc : norm;
 
     // ---- every CTA: level-1 histogram of its 1024 tokens, then into the global one ----
     for (int b = threadIdx.x; b < kBins; b += kSelThreads) {
@@ -428,7 +426,9 @@ select_kernel(int L, const float *__restrict__ acc, const float *__restrict__ no
     }
     if (threadIdx.x < 4) c.rng[threadIdx.x] = 0;
     grid_launch_dependents();
-    grid_dependency_wait();       // the scores are the previous kernel's output
+    grid_dependency_wait(acc, norm);   // the scores are the previous kernel's output
+    const float *bud = (mode & ZIPVL_BUDGET_BY_NORM) ? norm : acc;
+    const float *rank = (mode & ZIPVL_TOPK_BY_ACC) ? acc : norm;
     __syncthreads();
     // a single CTA (short sequences) walks the whole row and keeps the histogram in
     // shared memory; several CTAs take 1024 tokens each and meet in the global one
