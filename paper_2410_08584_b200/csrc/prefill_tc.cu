@@ -29,6 +29,9 @@
 // Tensor memory (512 columns): S_A | S_B | O_A | O_B, 128 fp32 columns each; P
 // aliases the first 64 columns of its S.  Every wait is bounded; a wait that
 // runs out sets ZIPVL_DEV_TIMEOUT and all roles unwind to the common exit.
+#include <stdlib.h>
+#include <string.h>
+
 #include <type_traits>
 
 #include "tc.cuh"
@@ -52,6 +55,9 @@ constexpr uint32_t kTmemCols = 512;
 // the running max may lag a tile's max by this many octaves before O is rescaled: P stays
 // below 2^32 (bfloat16 and fp32 carry that) or 2^8 (IEEE half tops out at 65504)
 constexpr float kRescaleThreshold = 32.0f, kRescaleThresholdHalf = 8.0f;
+// kept rows x query heads up to which the single-tile kernel is launched instead of this one
+// (0: never by default -- it measured slower at every size tried, see the dispatch below)
+constexpr long long kSingleTileMaxRows = 0;
 
 struct Barriers {
     uint64_t q_full;
@@ -595,6 +601,19 @@ zipvl_status launch_prefill_tc(const LayerArgs &a, const void *q, const void *k,
                                int out_mode, void *k_cache, void *v_cache, int capacity,
                                int32_t *len_out, void *ws, int32_t *status_word, cudaStream_t st) {
     (void)ws;
+    // The kernel with one 128-row query tile per CTA and two CTAs per SM (prefill_tc1.cu) has
+    // smaller work items and hides a CTA's prologue and epilogue behind its neighbour, but
+    // every key / value tile then feeds one query tile instead of two, and with room for
+    // only one K and one V buffer its loads (2500-3400 cycles per tile next to busy softmax
+    // warps) sit on the critical path of each step: 94 against 72 microseconds on the
+    // 2944-token, 32-head layer, 829 against 1147 TFLOP/s on the 18432-token one.  It gives
+    // the same bits and stays selectable with ZIPVL_PREFILL_KERNEL=single (pair = this one).
+    const char *env = getenv("ZIPVL_PREFILL_KERNEL");
+    const int forced = !env ? 0 : (!strcmp(env, "pair") ? 1 : (!strcmp(env, "single") ? 2 : 0));
+    const bool single = forced ? (forced == 2) : ((long long)k_max * a.Hq <= kSingleTileMaxRows);
+    if (single)
+        return launch_prefill_tc1(a, q, k, v, idx, k_dev, k_max, out, out_mode, k_cache, v_cache,
+                                  capacity, len_out, status_word, st);
     auto kernel = a.half ? prefill_tc_kernel<true> : prefill_tc_kernel<false>;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
     if (e != cudaSuccess)

@@ -197,6 +197,36 @@ def test_fused_prefill_and_compaction_equal_the_two_calls(zipvl, name, out_mode)
                                   oracle.compact_rows(layer.k.view(bits).numpy(), T))
 
 
+@pytest.mark.parametrize("name", ["llava7b_small_bf16", "video_gqa_small", "ragged_129", "llava7b_small_fp16",
+                                  "one_token"])
+@pytest.mark.parametrize("out_mode", ["padded", "compact"])
+def test_single_tile_attention_kernel_gives_the_bits_of_the_default_one(zipvl, name, out_mode, monkeypatch):
+    """The library's second tensor-core attention kernel (one 128-row query tile per thread
+    block, two blocks per SM; selected by an environment variable) does the same arithmetic in
+    the same order as the default one, which the tests above hold against the oracle: outputs,
+    compacted caches and lengths must agree bit for bit."""
+    layer = CASES[name]()
+    q, k, v, probe = put(layer)
+    desc = zipvl.layer_desc(q, k)
+    acc, norm = zipvl.zipvl_score(desc, q, k, probe)
+    k_dev, idx = zipvl.zipvl_select(acc, norm, layer.tau)
+    mode = zipvl.OUT_PADDED if out_mode == "padded" else zipvl.OUT_COMPACT
+    res = {}
+    for kernel in ("pair", "single"):
+        monkeypatch.setenv("ZIPVL_PREFILL_KERNEL", kernel)
+        st = status_word()
+        kc, vc = torch.zeros_like(k), torch.zeros_like(v)
+        out = torch.zeros((layer.L, layer.n_q_heads, layer.head_dim), dtype=q.dtype, device=DEV)
+        _, n = zipvl.zipvl_sparse_prefill_compact(desc, q, k, v, idx, k_dev, layer.L, kc, vc, layer.L,
+                                                  out=out, out_mode=mode, status=st)
+        torch.cuda.synchronize()
+        assert st.item() == 0
+        res[kernel] = (out, kc, vc, int(n.item()))
+    a, b = res["pair"], res["single"]
+    assert a[3] == b[3] == int(k_dev.item())
+    assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1]) and torch.equal(a[2], b[2])
+
+
 def test_fused_prefill_compaction_reports_a_small_cache(zipvl):
     layer = CASES["llava7b_small_bf16"]()
     q, k, v, probe = put(layer)
