@@ -157,7 +157,8 @@ zipvl_status zipvl_score(const zipvl_layer *layer, const void *q, const void *k,
  * together; any other bit is ZIPVL_ERR_INVALID_ARG.
  *
  * acc, norm: device float[L], non-negative; a negative or NaN entry counts as zero in
- * the sums, ranks by its bit pattern and is reported as ZIPVL_DEV_BAD_VALUE.
+ * the sums, ranks by its bit pattern and is reported as ZIPVL_DEV_BAD_VALUE.  Sums are
+ * exact for scores below 2^18 (a column sum of attention is at most n_probe x n_q_heads).
  * k_out: device int32[1].
  * idx: device int32[L].  kept_mass: device float[1] or NULL.
  * ws: zipvl_workspace_bytes(ZIPVL_OP_SELECT).  L <= 2^20.
@@ -306,6 +307,21 @@ zipvl_status zipvl_prefill_layer_host(const zipvl_layer *layer, const void *q, c
                                       const void *v, const int32_t *probe_pos, int32_t n_probe,
                                       float tau, int32_t *k_out, int32_t *idx_out, void *out,
                                       void *k_cache_out, void *v_cache_out);
+
+/*
+ * zipvl_layer_step_host -- zipvl_prefill_layer_host followed by one decode step, from HOST
+ * buffers: Algorithm 1 for the layer, then Algorithm 2 for one new token on the cache the
+ * call has just compacted (the new key / value are appended behind the kept rows, Eq. 4,
+ * and the new query attends over all of them, Eq. 5).  q_new: [Hq,d]; k_new, v_new:
+ * [Hkv,d]; decode_out: [Hq,d]; all HOST, all four given or all four NULL (then this is
+ * zipvl_prefill_layer_host).  The caches copied back hold the kept rows, not the appended
+ * one.  At most 8 query heads per KV head, as for zipvl_decode.
+ */
+zipvl_status zipvl_layer_step_host(const zipvl_layer *layer, const void *q, const void *k,
+                                   const void *v, const int32_t *probe_pos, int32_t n_probe,
+                                   float tau, int32_t *k_out, int32_t *idx_out, void *out,
+                                   void *k_cache_out, void *v_cache_out, const void *q_new,
+                                   const void *k_new, const void *v_new, void *decode_out);
 
 /*
  * zipvl_release_host_scratch -- give back the device memory zipvl_prefill_layer_host

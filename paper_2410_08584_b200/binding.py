@@ -25,7 +25,7 @@ EXPORTS = ["zipvl_status_string", "zipvl_last_error", "zipvl_version", "zipvl_la
            "zipvl_workspace_bytes",
            "zipvl_score", "zipvl_select", "zipvl_sparse_prefill", "zipvl_compact_kv",
            "zipvl_sparse_prefill_compact",
-           "zipvl_decode", "zipvl_decode_noalloc", "zipvl_prefill_layer_host",
+           "zipvl_decode", "zipvl_decode_noalloc", "zipvl_prefill_layer_host", "zipvl_layer_step_host",
            "zipvl_release_host_scratch", "zipvl_selftest_wait_timeout"]
 
 
@@ -89,6 +89,8 @@ def load():
                                          vp, i32, vp, vp, vp]
     lib.zipvl_prefill_layer_host.restype = C.c_int
     lib.zipvl_prefill_layer_host.argtypes = [lp, vp, vp, vp, vp, i32, f32, vp, vp, vp, vp, vp]
+    lib.zipvl_layer_step_host.restype = C.c_int
+    lib.zipvl_layer_step_host.argtypes = [lp, vp, vp, vp, vp, i32, f32, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.zipvl_selftest_wait_timeout.restype = C.c_int
     lib.zipvl_selftest_wait_timeout.argtypes = [i32, vp, vp, vp]
     _lib = lib
@@ -291,6 +293,28 @@ def zipvl_selftest_wait_timeout(poll_limit, progress, status, stream=None):
     _dev(progress, "progress", torch.int32), _dev(status, "status", torch.int32)
     _check(load().zipvl_selftest_wait_timeout(int(poll_limit), _ptr(progress), _ptr(status),
                                               _stream(stream)))
+
+
+def zipvl_layer_step_host(layer, q, k, v, probe_pos, tau, q_new, k_new, v_new, out=None, k_cache=None,
+                          v_cache=None, idx=None, decode_out=None):
+    """Algorithm 1 for the layer and one decode step (Algorithm 2) on the cache it leaves,
+    from HOST tensors.  Returns (k, idx, out, k_cache, v_cache, decode_out) as host tensors."""
+    for t in (q, k, v, probe_pos, q_new, k_new, v_new):
+        if t.is_cuda or not t.is_contiguous():
+            raise ValueError("zipvl_layer_step_host takes contiguous host tensors")
+    pin = q.is_pinned()
+    mk = lambda shape, dt: torch.empty(shape, dtype=dt, pin_memory=pin)
+    out = mk(q.shape, q.dtype) if out is None else out
+    k_cache = mk(k.shape, k.dtype) if k_cache is None else k_cache
+    v_cache = mk(v.shape, v.dtype) if v_cache is None else v_cache
+    idx = mk((layer.L,), torch.int32) if idx is None else idx
+    decode_out = mk(q_new.shape, q_new.dtype) if decode_out is None else decode_out
+    kk = C.c_int32(0)
+    _check(load().zipvl_layer_step_host(C.byref(layer), _ptr(q), _ptr(k), _ptr(v), _ptr(probe_pos),
+                                        probe_pos.numel(), float(tau), C.cast(C.byref(kk), C.c_void_p),
+                                        _ptr(idx), _ptr(out), _ptr(k_cache), _ptr(v_cache), _ptr(q_new),
+                                        _ptr(k_new), _ptr(v_new), _ptr(decode_out)))
+    return kk.value, idx, out, k_cache, v_cache, decode_out
 
 
 def zipvl_prefill_layer_host(layer, q, k, v, probe_pos, tau, out=None, k_cache=None, v_cache=None,

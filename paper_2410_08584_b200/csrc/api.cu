@@ -314,30 +314,49 @@ zipvl_status zipvl_prefill_layer_host(const zipvl_layer *layer, const void *q, c
                                       const void *v, const int32_t *probe_pos, int32_t n_probe,
                                       float tau, int32_t *k_out, int32_t *idx_out, void *out,
                                       void *k_cache_out, void *v_cache_out) {
+    return zipvl_layer_step_host(layer, q, k, v, probe_pos, n_probe, tau, k_out, idx_out, out,
+                                 k_cache_out, v_cache_out, nullptr, nullptr, nullptr, nullptr);
+}
+
+zipvl_status zipvl_layer_step_host(const zipvl_layer *layer, const void *q, const void *k,
+                                   const void *v, const int32_t *probe_pos, int32_t n_probe,
+                                   float tau, int32_t *k_out, int32_t *idx_out, void *out,
+                                   void *k_cache_out, void *v_cache_out, const void *q_new,
+                                   const void *k_new, const void *v_new, void *decode_out) {
     LayerArgs a{};
-    zipvl_status st_ = check_layer("zipvl_prefill_layer_host", layer, &a);
+    zipvl_status st_ = check_layer("zipvl_layer_step_host", layer, &a);
     if (st_ != ZIPVL_OK) return st_;
     if (!q || !k || !v || !probe_pos || n_probe < 1)
-        return fail(ZIPVL_ERR_INVALID_ARG, "zipvl_prefill_layer_host: NULL input or n_probe < 1");
+        return fail(ZIPVL_ERR_INVALID_ARG, "zipvl_layer_step_host: NULL input or n_probe < 1");
     if (layer->q_stride_tok || layer->kv_stride_tok)
-        return fail(ZIPVL_ERR_UNSUPPORTED, "zipvl_prefill_layer_host: contiguous tensors only");
+        return fail(ZIPVL_ERR_UNSUPPORTED, "zipvl_layer_step_host: contiguous tensors only");
+    const bool with_decode = (q_new != nullptr);
+    if (with_decode && (!k_new || !v_new || !decode_out))
+        return fail(ZIPVL_ERR_INVALID_ARG, "zipvl_layer_step_host: the decode step needs q_new, k_new, v_new and decode_out");
+    if (with_decode && a.G > 8)
+        return fail(ZIPVL_ERR_UNSUPPORTED, "zipvl_layer_step_host: more than 8 query heads per kv head");
     const size_t eb = elem_bytes(layer->dtype);
     const size_t qb = (size_t)a.L * a.Hq * a.D * eb, kb = (size_t)a.L * a.Hkv * a.D * eb;
     const size_t ws_score = zipvl_workspace_bytes(ZIPVL_OP_SCORE, layer, n_probe, 1);
     const size_t ws_pf = zipvl_workspace_bytes(ZIPVL_OP_SPARSE_PREFILL, layer, 0, 1);
     size_t ws_b = ws_score > ws_pf ? ws_score : ws_pf;
     if (ws_b < select_ws_bytes()) ws_b = select_ws_bytes();
+    // the decode step runs on the cache this call has just compacted: capacity L + 1 rows
+    const size_t ws_dec = with_decode ? align256(decode_ws_bytes(1, a.Hq, a.D, a.L + 1)) : 0;
+    if (ws_b < ws_dec) ws_b = ws_dec;
+    const size_t qn_b = (size_t)a.Hq * a.D * eb, kn_b = (size_t)a.Hkv * a.D * eb;
     // one stream-ordered allocation carved into pieces
     size_t off = 0;
     auto carve = [&](size_t bytes) { size_t o = off; off += align256(bytes); return o; };
     const size_t o_q = carve(qb), o_k = carve(kb), o_v = carve(kb), o_out = carve(qb),
-                 o_kc = carve(kb), o_vc = carve(kb), o_probe = carve((size_t)n_probe * 4),
+                 o_kc = carve(kb + kn_b), o_vc = carve(kb + kn_b), o_probe = carve((size_t)n_probe * 4),
+                 o_qn = carve(qn_b), o_kn = carve(kn_b), o_vn = carve(kn_b), o_dec = carve(qn_b),
                  o_acc = carve((size_t)a.L * 4), o_norm = carve((size_t)a.L * 4),
                  o_idx = carve((size_t)a.L * 4), o_misc = carve(256), o_ws = carve(ws_b);
     char *base = nullptr;
     cudaStream_t s = nullptr;
     cudaMemPool_t pool = nullptr;
-    int32_t misc[4] = {0, 0, 0, 0};
+    int32_t misc[4] = {0, 0, 0, 0};   // k, cache length, device status word, (cache capacity)
     ZIPVL_CUDA(cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking));
     ZIPVL_CUDA(host_pool(&pool));
     ZIPVL_CUDA(cudaMallocFromPoolAsync((void **)&base, off, pool, s));
@@ -348,6 +367,11 @@ zipvl_status zipvl_prefill_layer_host(const zipvl_layer *layer, const void *q, c
         ZIPVL_CUDA(cudaMemcpyAsync(base + o_k, k, kb, cudaMemcpyHostToDevice, s));
         ZIPVL_CUDA(cudaMemcpyAsync(base + o_v, v, kb, cudaMemcpyHostToDevice, s));
         ZIPVL_CUDA(cudaMemcpyAsync(base + o_probe, probe_pos, (size_t)n_probe * 4, cudaMemcpyHostToDevice, s));
+        if (with_decode) {
+            ZIPVL_CUDA(cudaMemcpyAsync(base + o_qn, q_new, qn_b, cudaMemcpyHostToDevice, s));
+            ZIPVL_CUDA(cudaMemcpyAsync(base + o_kn, k_new, kn_b, cudaMemcpyHostToDevice, s));
+            ZIPVL_CUDA(cudaMemcpyAsync(base + o_vn, v_new, kn_b, cudaMemcpyHostToDevice, s));
+        }
         st_ = zipvl_score(layer, base + o_q, base + o_k, (int32_t *)(base + o_probe), n_probe,
                           (float *)(base + o_acc), (float *)(base + o_norm), nullptr, base + o_ws,
                           ws_b, d_misc + 2, s);
@@ -360,6 +384,18 @@ zipvl_status zipvl_prefill_layer_host(const zipvl_layer *layer, const void *q, c
                                            ZIPVL_OUT_PADDED, base + o_kc, base + o_vc, a.L, d_misc + 1,
                                            base + o_ws, ws_b, d_misc + 2, s);
         if (st_ != ZIPVL_OK) goto done;
+        if (with_decode) {
+            // Algorithm 2 on the cache just built: d_misc[1] holds its length, d_misc[3] its
+            // capacity, d_misc + 4 (8-byte aligned) the one request's offset 0
+            const int32_t cap = a.L + 1;
+            ZIPVL_CUDA(cudaMemcpyAsync(d_misc + 3, &cap, 4, cudaMemcpyHostToDevice, s));
+            zipvl_decode_desc dd = {1, a.Hq, a.Hkv, a.D, layer->dtype, layer->softmax_scale};
+            st_ = zipvl_decode(&dd, base + o_qn, base + o_kn, base + o_vn, base + o_kc, base + o_vc,
+                               (const int64_t *)(d_misc + 4), d_misc + 3, d_misc + 1, cap, base + o_dec,
+                               base + o_ws, ws_b, d_misc + 2, s);
+            if (st_ != ZIPVL_OK) goto done;
+            ZIPVL_CUDA(cudaMemcpyAsync(decode_out, base + o_dec, qn_b, cudaMemcpyDeviceToHost, s));
+        }
         ZIPVL_CUDA(cudaMemcpyAsync(misc, d_misc, sizeof(misc), cudaMemcpyDeviceToHost, s));
         if (out) ZIPVL_CUDA(cudaMemcpyAsync(out, base + o_out, qb, cudaMemcpyDeviceToHost, s));
         if (idx_out) ZIPVL_CUDA(cudaMemcpyAsync(idx_out, base + o_idx, (size_t)a.L * 4, cudaMemcpyDeviceToHost, s));

@@ -8,9 +8,10 @@
 //            tau * S; p = #{a > v*} + the number of copies of v* still needed;
 //   top-p    the p-th largest ranking score u*; ties at u* go to the smaller
 //            position.
-// Rows of up to 4096 tokens: one CTA histograms the whole row on the top 12 key
-// bits (count and sum of the budget score, count of the ranking score) in shared
-// memory.  Longer rows: ceil(L / 1024) CTAs histogram 1024 tokens each, add their
+// Rows of up to 4096 tokens run on one CTA that holds the row in registers (see
+// select_solo_kernel further down).  Longer rows: ceil(L / 1024) CTAs histogram 1024
+// tokens each on the top 12 key bits (count and sum of the budget score, count of the
+// ranking score), add their
 // non-empty bins to a global histogram (64 KB of the workspace, cleared by a memset
 // node in front of the kernel) and the last CTA to finish (ticket) goes on alone.
 // That CTA finds the crossing bin (one warp scans the occupied bin range), refines
@@ -430,12 +431,9 @@ select_kernel(int L, const float *__restrict__ acc, const float *__restrict__ no
     const float *bud = (mode & ZIPVL_BUDGET_BY_NORM) ? norm : acc;
     const float *rank = (mode & ZIPVL_TOPK_BY_ACC) ? acc : norm;
     __syncthreads();
-    // a single CTA (short sequences) walks the whole row and keeps the histogram in
-    // shared memory; several CTAs take 1024 tokens each and meet in the global one
-    const bool solo = (gridDim.x == 1);
-    unsigned long long my_sum = 0;                 // this thread's share of S (used when solo)
+    // every CTA takes 1024 tokens; they meet in the global histogram
     bool bad_value = false;                        // a score that is negative or not a number
-    const int row_end = solo ? L : min(L, (int)(blockIdx.x + 1) * kSelThreads);
+    const int row_end = min(L, (int)(blockIdx.x + 1) * kSelThreads);
     for (int jb = blockIdx.x * kSelThreads; jb < row_end; jb += kSelThreads * kBatch) {
         float vbs[kBatch], vrs[kBatch];            // the loads of a batch are in flight together
 #pragma unroll
@@ -449,7 +447,6 @@ select_kernel(int L, const float *__restrict__ acc, const float *__restrict__ no
             if (jb + u * kSelThreads >= row_end) break;   // (the same for every thread)
             const bool act = jb + u * kSelThreads + (int)threadIdx.x < row_end;
             const unsigned long long fxb = act ? to_fx(vbs[u]) : 0ull;
-            my_sum += fxb;
             bad_value |= act && (!(vbs[u] >= 0.f) || !(vrs[u] >= 0.f));
             hist_add(sm.cnt_b, &sm, act, float_key(vbs[u]) >> 20, fxb, &c.rng[0]);
             hist_add(sm.cnt_r, nullptr, act, float_key(vrs[u]) >> 20, 0ull, &c.rng[2]);
@@ -459,7 +456,6 @@ select_kernel(int L, const float *__restrict__ acc, const float *__restrict__ no
     // still completes, the caller is told)
     if (bad_value) report(status_word, ZIPVL_DEV_BAD_VALUE);
     __syncthreads();
-    if (!solo) {
     for (int b = threadIdx.x; b < kBins; b += kSelThreads) {
         const unsigned int cb = sm.cnt_b[b], cr = sm.cnt_r[b];
         if (cb) {
@@ -488,7 +484,6 @@ select_kernel(int L, const float *__restrict__ acc, const float *__restrict__ no
     }
     if (threadIdx.x < 4) c.rng[threadIdx.x] = __ldcg(&gh->rng[threadIdx.x]);
     __syncthreads();
-    }
 
     // ---- the budget p (Eq. 7), then the threshold of the ranking score: the p-th
     // largest (Eq. 9).  Both are the same descent (by cumulative sum over the budget
@@ -504,11 +499,8 @@ select_kernel(int L, const float *__restrict__ acc, const float *__restrict__ no
         const float *x = by_sum ? bud : rank;
         unsigned long long target = p;
         if (by_sum) {
-            unsigned long long part = my_sum;
-            if (!solo) {
-                part = 0;
-                for (int b = threadIdx.x; b < kBins; b += kSelThreads) part += bin_sum64(sm, b);
-            }
+            unsigned long long part = 0;
+            for (int b = threadIdx.x; b < kBins; b += kSelThreads) part += bin_sum64(sm, b);
             const unsigned long long S_b = block_sum64(part, c);
             target = (unsigned long long)ceil((double)tau * (double)S_b);
         }
@@ -612,6 +604,417 @@ select_kernel(int L, const float *__restrict__ acc, const float *__restrict__ no
     }
 }
 
+
+// ---------------------------------------------------------------------------------------
+// Rows of up to 4096 tokens: one CTA of 256 threads with the whole row in registers.
+//
+// Thread t owns positions 16t .. 16t+15 (four 16-byte loads per score vector), so the row is
+// read from memory once and the ascending emission is a walk over the thread's own registers.
+// A block-wide step costs a barrier plus its warp shuffles once per warp, so the CTA is kept
+// to eight warps and every phase to a few such steps; nothing loops over the row.
+//
+// The threshold searches are the ones described at the top of the file, with one change that
+// matters at this size: the histogram levels adapt to the data.  Level 1 spreads its 4096
+// bins over [smallest key, largest key] of the row instead of over the top 12 key bits (scores
+// of one layer lie within a few octaves of each other, which is a few dozen of the fixed
+// bins), so the crossing bin holds a handful of tokens instead of hundreds; each further
+// level spreads 4096 bins over the crossing bin of the level before.  The descent ends when a
+// bin holds one token or spans one key value (ties): two levels as a rule, three at most.
+// ---------------------------------------------------------------------------------------
+#ifndef ZIPVL_SOLO_THREADS
+#define ZIPVL_SOLO_THREADS 512
+#endif
+constexpr int kSoloThreads = ZIPVL_SOLO_THREADS;
+constexpr int kSoloPer = kSoloMax / kSoloThreads;   // 16 positions per thread
+constexpr int kSoloWarps = kSoloThreads / 32;
+
+struct SoloSmem {                      // dynamic shared memory
+    // fixed-point sum of the budget score per bin as three words of 16-bit pieces (bits 0-15,
+    // 16-31, 32 and up of each addend): three independent 32-bit adds without a carry to pass
+    // on; exact while a bin's pieces stay below 2^32, i.e. for scores below 2^18
+    unsigned int sum16[3][kBins];
+    unsigned int cnt[kBins];
+    unsigned int cnt_r[kBins];         // level 1 of the ranking score (filled in the same walk)
+};
+__device__ __forceinline__ void solo_add(SoloSmem &sm, unsigned int d, unsigned long long fx) {
+    atomicAdd(&sm.cnt[d], 1u);
+    atomicAdd(&sm.sum16[0][d], (unsigned int)fx & 0xffffu);
+    atomicAdd(&sm.sum16[1][d], ((unsigned int)fx >> 16));
+    atomicAdd(&sm.sum16[2][d], (unsigned int)(fx >> 32));
+}
+__device__ __forceinline__ unsigned long long solo_sum(const SoloSmem &sm, int b) {
+    return (unsigned long long)sm.sum16[0][b] + ((unsigned long long)sm.sum16[1][b] << 16) +
+           ((unsigned long long)sm.sum16[2][b] << 32);
+}
+struct SoloCtl {                       // static shared memory
+    unsigned long long wsum[kSoloWarps], sum_gt, bin_sum;
+    unsigned int wcnt[kSoloWarps], wmin[2][kSoloWarps], wmax[2][kSoloWarps];
+    unsigned int hit, hit_bin, cnt_gt, bin_cnt, one_key;
+};
+
+// block-wide (256 threads) exclusive prefix of a (count, sum) pair in thread order, and totals
+__device__ __forceinline__ void solo_scan(unsigned int vc, unsigned long long vs, SoloCtl &c,
+                                          unsigned int *pc, unsigned long long *ps,
+                                          unsigned int *tc = nullptr, unsigned long long *ts = nullptr) {
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    unsigned int ic = vc;
+    unsigned long long is = vs;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const unsigned int nc = __shfl_up_sync(0xffffffffu, ic, o);
+        const unsigned long long ns = __shfl_up_sync(0xffffffffu, is, o);
+        if (lane >= o) { ic += nc; is += ns; }
+    }
+    __syncthreads();                                   // earlier readers of wcnt / wsum are done
+    if (lane == 31) { c.wcnt[w] = ic; c.wsum[w] = is; }
+    __syncthreads();
+    unsigned int bc = 0, allc = 0;
+    unsigned long long bs = 0, alls = 0;
+#pragma unroll
+    for (int i = 0; i < kSoloWarps; ++i) {
+        const unsigned int wc = c.wcnt[i];
+        const unsigned long long wsm = c.wsum[i];
+        if (i < w) { bc += wc; bs += wsm; }
+        allc += wc; alls += wsm;
+    }
+    *pc = bc + ic - vc;
+    *ps = bs + is - vs;
+    if (tc) *tc = allc;
+    if (ts) *ts = alls;
+}
+
+// One adaptive histogram level below the first: the range is the crossing bin of the level
+// before, [base, base + 2^width_log2); a token whose key lies in it falls into bin
+// (key - base) >> shift.
+__device__ __forceinline__ bool solo_bin(unsigned int key, unsigned int base, int width_log2, int shift,
+                                         unsigned int *d) {
+    const unsigned int off = key - base;
+    *d = off >> shift;
+    return key >= base && (off >> width_log2) == 0u;
+}
+
+// The crossing bin from the top.  by_sum: first non-empty bin at which carry_sum + descending
+// cumulative sum >= target; else the same by count.  Publishes hit (0xffffffff: none),
+// hit_bin, cnt_gt / sum_gt (everything above the bin, carries included), bin_cnt / bin_sum.
+// Three steps, each behind one barrier, so that only the warp that holds the crossing does
+// the fine search: (1) every warp adds up its bins (kBins / warps, from the top), (2) warp 0
+// walks the warp totals to the warp where the running total crosses, (3) that warp scans its
+// lanes and the lane that crosses walks its own bins.
+__device__ void solo_find_bin(const SoloSmem &sm, bool by_sum, unsigned long long target,
+                              unsigned int carry_cnt, unsigned long long carry_sum, SoloCtl &c) {
+    constexpr int kPer = kBins / kSoloThreads;         // bins per thread
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const int b_top = kBins - 1 - (int)threadIdx.x * kPer;   // my bins: b_top, b_top-1, ...
+    unsigned int cb[kPer];
+    unsigned int lc = 0;
+#pragma unroll
+    for (int v4 = 0; v4 < kPer / 4; ++v4) {
+        const uint4 q = *reinterpret_cast<const uint4 *>(&sm.cnt[b_top - 3 - 4 * v4]);
+        cb[4 * v4 + 0] = q.w; cb[4 * v4 + 1] = q.z; cb[4 * v4 + 2] = q.y; cb[4 * v4 + 3] = q.x;
+        lc += q.x + q.y + q.z + q.w;
+    }
+    unsigned long long ls = 0;
+    if (by_sum && lc) {
+#pragma unroll
+        for (int i = 0; i < kPer; ++i)
+            if (cb[i]) ls += solo_sum(sm, b_top - i);
+    }
+    // (1) warp totals: the count in one instruction, the sum as three 20-bit pieces
+    const unsigned int wc = __reduce_add_sync(0xffffffffu, lc);
+    unsigned long long wsum = 0;
+    if (by_sum) {
+        wsum = (unsigned long long)__reduce_add_sync(0xffffffffu, (unsigned int)ls & 0xfffffu) +
+               ((unsigned long long)__reduce_add_sync(0xffffffffu, (unsigned int)(ls >> 20) & 0xfffffu) << 20) +
+               ((unsigned long long)__reduce_add_sync(0xffffffffu, (unsigned int)(ls >> 40)) << 40);
+    }
+    __syncthreads();                                   // earlier readers of wcnt / wsum / hit are done
+    if (lane == 0) { c.wcnt[w] = wc; c.wsum[w] = wsum; }
+    __syncthreads();
+    // (2) the warp in which the running total crosses
+    if (threadIdx.x == 0) {
+        unsigned int run_c = carry_cnt;
+        unsigned long long run_s = carry_sum;
+        unsigned int hit_w = 0xffffffffu;
+        for (int i = 0; i < kSoloWarps; ++i) {
+            const unsigned int tc = c.wcnt[i];
+            const unsigned long long ts = c.wsum[i];
+            const bool ok = tc > 0 && (by_sum ? (run_s + ts >= target) : ((unsigned long long)run_c + tc >= target));
+            if (ok) { hit_w = i; break; }
+            run_c += tc; run_s += ts;
+        }
+        c.hit = hit_w;                                 // (0xffffffff: no bin qualifies)
+        c.cnt_gt = run_c;                              // everything above that warp's bins
+        c.sum_gt = run_s;
+    }
+    __syncthreads();
+    // (3) inside that warp
+    if ((unsigned int)w == c.hit) {
+        unsigned int ic = lc;
+        unsigned long long is = ls;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const unsigned int nc = __shfl_up_sync(0xffffffffu, ic, o);
+            const unsigned long long ns = __shfl_up_sync(0xffffffffu, is, o);
+            if (lane >= o) { ic += nc; is += ns; }
+        }
+        unsigned int run_c = c.cnt_gt + ic - lc;
+        unsigned long long run_s = c.sum_gt + is - ls;
+        const bool mine = lc > 0 && (by_sum ? (run_s + ls >= target) : ((unsigned long long)run_c + lc >= target));
+        const unsigned int who = __ballot_sync(0xffffffffu, mine);
+        if (who && lane == __ffs(who) - 1) {           // the first lane (highest bins) that crosses
+#pragma unroll
+            for (int i = 0; i < kPer; ++i) {
+                if (cb[i]) {
+                    const unsigned long long sb = by_sum ? solo_sum(sm, b_top - i) : 0ull;
+                    const bool ok = by_sum ? (run_s + sb >= target) : ((unsigned long long)run_c + cb[i] >= target);
+                    if (ok) {
+                        c.cnt_gt = run_c;
+                        c.sum_gt = run_s;
+                        c.bin_cnt = cb[i];
+                        c.bin_sum = sb;
+                        c.hit_bin = (unsigned int)(b_top - i);
+                        break;
+                    }
+                    run_c += cb[i]; run_s += sb;
+                }
+            }
+        }
+    }
+    __syncthreads();
+}
+
+template <bool kKeepLast>
+__global__ void __launch_bounds__(kSoloThreads)
+select_solo_kernel(int L, const float *__restrict__ acc, const float *__restrict__ norm, float tau,
+                   uint32_t mode, int fixed_k, int32_t *__restrict__ k_out, int32_t *__restrict__ idx,
+                   float *__restrict__ kept_mass, int32_t *status_word) {
+    extern __shared__ __align__(16) unsigned char sel_dyn[];
+    SoloSmem &sm = *reinterpret_cast<SoloSmem *>(sel_dyn);
+    __shared__ SoloCtl c;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    auto clear = [&](void *p, int bytes) {
+        uint4 *z = reinterpret_cast<uint4 *>(p);
+        for (int e = threadIdx.x; e < bytes / 16; e += kSoloThreads) z[e] = make_uint4(0, 0, 0, 0);
+    };
+    clear(&sm, sizeof(SoloSmem));      // while the previous kernel may still be running
+    grid_launch_dependents();
+    grid_dependency_wait(acc, norm);   // the scores are the previous kernel's output
+    const bool bud_is_norm = (mode & ZIPVL_BUDGET_BY_NORM) != 0, rank_is_acc = (mode & ZIPVL_TOPK_BY_ACC) != 0;
+    // ---- the row into registers: positions j0 .. j0+15 (a vector that is not 16-byte aligned
+    // is read element by element) ----
+    const int j0 = (int)threadIdx.x * kSoloPer;
+    float av[kSoloPer], nv[kSoloPer];
+    const bool vec = (((uintptr_t)acc | (uintptr_t)norm) & 15u) == 0;
+#pragma unroll
+    for (int v4 = 0; v4 < kSoloPer / 4; ++v4) {
+        const int j = j0 + 4 * v4;
+        if (vec && j + 4 <= L) {
+            const float4 a4 = *reinterpret_cast<const float4 *>(acc + j);
+            const float4 n4 = *reinterpret_cast<const float4 *>(norm + j);
+            av[4 * v4] = a4.x; av[4 * v4 + 1] = a4.y; av[4 * v4 + 2] = a4.z; av[4 * v4 + 3] = a4.w;
+            nv[4 * v4] = n4.x; nv[4 * v4 + 1] = n4.y; nv[4 * v4 + 2] = n4.z; nv[4 * v4 + 3] = n4.w;
+        } else {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                av[4 * v4 + e] = (j + e < L) ? acc[j + e] : 0.f;
+                nv[4 * v4 + e] = (j + e < L) ? norm[j + e] : 0.f;
+            }
+        }
+    }
+    // keys of the two scores, their ranges over the row, S of the budget score
+    unsigned int kb[kSoloPer], kr[kSoloPer];
+    unsigned int mn[2] = {0xffffffffu, 0xffffffffu}, mx[2] = {0u, 0u};
+    unsigned long long my_sum = 0;
+    bool bad_value = false;
+#pragma unroll
+    for (int e = 0; e < kSoloPer; ++e) {
+        const float vb = bud_is_norm ? nv[e] : av[e], vr = rank_is_acc ? av[e] : nv[e];
+        kb[e] = float_key(vb);
+        kr[e] = float_key(vr);
+        if (j0 + e < L) {
+            mn[0] = min(mn[0], kb[e]); mx[0] = max(mx[0], kb[e]);
+            mn[1] = min(mn[1], kr[e]); mx[1] = max(mx[1], kr[e]);
+            my_sum += to_fx(vb);
+            bad_value |= !(vb >= 0.f) || !(vr >= 0.f);
+        }
+    }
+    if (bad_value) report(status_word, ZIPVL_DEV_BAD_VALUE);
+#pragma unroll
+    for (int x = 0; x < 2; ++x) {
+        mn[x] = __reduce_min_sync(0xffffffffu, mn[x]);
+        mx[x] = __reduce_max_sync(0xffffffffu, mx[x]);
+        if (lane == 0) { c.wmin[x][warp] = mn[x]; c.wmax[x][warp] = mx[x]; }
+    }
+    __syncthreads();                   // the ranges are in; the histograms are clear
+#pragma unroll
+    for (int x = 0; x < 2; ++x) {
+        mn[x] = 0xffffffffu; mx[x] = 0u;
+#pragma unroll
+        for (int i = 0; i < kSoloWarps; ++i) { mn[x] = min(mn[x], c.wmin[x][i]); mx[x] = max(mx[x], c.wmax[x][i]); }
+    }
+    auto first_shift = [](unsigned int lo, unsigned int hi) {
+        const int bits = 32 - __clz(hi - lo);          // bits of the span (0 when all keys are equal)
+        return bits > 12 ? bits - 12 : 0;
+    };
+    const bool need_budget = !(fixed_k > 0) && (tau < 1.0f);
+    // ---- level 1 of both searches in one walk over the registers ----
+    const int shift1[2] = {first_shift(mn[0], mx[0]), first_shift(mn[1], mx[1])};
+#pragma unroll
+    for (int e = 0; e < kSoloPer; ++e) {
+        if (j0 + e < L) {
+            if (need_budget) {
+                solo_add(sm, (kb[e] - mn[0]) >> shift1[0], to_fx(bud_is_norm ? nv[e] : av[e]));
+            }
+            atomicAdd(&sm.cnt_r[(kr[e] - mn[1]) >> shift1[1]], 1u);
+        }
+    }
+    unsigned int p = (fixed_k > 0) ? (unsigned int)min(fixed_k, L) : (unsigned int)L;
+    unsigned int thr_key = 0, need_eq = L;
+#pragma unroll 1
+    for (int pass = need_budget ? 0 : 1; pass < 2; ++pass) {
+        const bool by_sum = (pass == 0);
+        if (!by_sum && p >= (unsigned int)L) break;
+        const unsigned int *keys = by_sum ? kb : kr;
+        unsigned long long target = p;
+        if (by_sum) {
+            unsigned int uc;
+            unsigned long long us, S_b;
+            solo_scan(0u, my_sum, c, &uc, &us, nullptr, &S_b);
+            target = (unsigned long long)ceil((double)tau * (double)S_b);
+        }
+        unsigned int base = mn[pass], carry_c = 0;
+        unsigned long long carry_s = 0;
+        int shift = shift1[pass], width_log2 = 32;
+        bool found = true;
+        if (!by_sum) {
+            // the ranking level 1 was counted into cnt_r: bring it to where the search reads
+            __syncthreads();
+            for (int e = threadIdx.x; e < kBins / 4; e += kSoloThreads)
+                reinterpret_cast<uint4 *>(sm.cnt)[e] = reinterpret_cast<const uint4 *>(sm.cnt_r)[e];
+        }
+#pragma unroll 1
+        for (int level = 0;; ++level) {
+            if (level > 0) {
+                // the next level: 4096 bins over the crossing bin of the one before
+                __syncthreads();
+                clear(sm.cnt, sizeof(sm.cnt));
+                if (by_sum) clear(sm.sum16, sizeof(sm.sum16));
+                __syncthreads();
+#pragma unroll
+                for (int e = 0; e < kSoloPer; ++e) {
+                    unsigned int d;
+                    if (j0 + e < L && solo_bin(keys[e], base, width_log2, shift, &d)) {
+                        if (by_sum) solo_add(sm, d, to_fx(bud_is_norm ? nv[e] : av[e]));
+                        else atomicAdd(&sm.cnt[d], 1u);
+                    }
+                }
+            }
+            __syncthreads();
+            solo_find_bin(sm, by_sum, target, carry_c, carry_s, c);
+            if (c.hit == 0xffffffffu) { found = false; break; }     // (rounding let no prefix qualify)
+            if (shift == 0) { thr_key = base + c.hit_bin; break; }  // the bin is one key value
+            if (c.bin_cnt == 1) {
+                // one token: its owner says which key it is
+#pragma unroll
+                for (int e = 0; e < kSoloPer; ++e) {
+                    unsigned int d;
+                    const bool in = (level == 0) ? (d = (keys[e] - base) >> shift, true)
+                                                 : solo_bin(keys[e], base, width_log2, shift, &d);
+                    if (j0 + e < L && in && d == c.hit_bin) c.one_key = keys[e];
+                }
+                __syncthreads();
+                thr_key = c.one_key;
+                break;
+            }
+            base += c.hit_bin << shift;
+            carry_c = c.cnt_gt;
+            carry_s = c.sum_gt;
+            width_log2 = shift;                        // (1..20: a bin of this level)
+            shift = shift > 12 ? shift - 12 : 0;
+        }
+        if (by_sum) {
+            if (found) {
+                // copies of the threshold value enter one at a time
+                const unsigned long long v = c.bin_cnt ? c.bin_sum / c.bin_cnt : 0ull;
+                unsigned long long need = 1;
+                if (target > c.sum_gt && v > 0) need = (target - c.sum_gt + v - 1) / v;
+                if (need < 1) need = 1;
+                if (need > c.bin_cnt) need = c.bin_cnt;
+                p = c.cnt_gt + (unsigned int)need;
+            }
+            thr_key = 0;
+        } else {
+            need_eq = p - c.cnt_gt;
+        }
+    }
+    __syncthreads();
+
+    // ---- emit T ascending from the registers ----
+    const bool all_sel = (p >= (unsigned int)L);
+    unsigned int n_gt = 0, n_eq = 0;
+#pragma unroll
+    for (int e = 0; e < kSoloPer; ++e) {
+        if (j0 + e < L) {
+            n_gt += kr[e] > thr_key;
+            n_eq += kr[e] == thr_key;
+        }
+    }
+    unsigned int eq_before;
+    unsigned long long gt_before;
+    solo_scan(n_eq, (unsigned long long)n_gt, c, &eq_before, &gt_before);
+    const unsigned int eq_take = all_sel ? n_eq : min(n_eq, need_eq > eq_before ? need_eq - eq_before : 0u);
+    unsigned int out = all_sel ? (unsigned int)min(j0, L) : (unsigned int)gt_before + min(eq_before, need_eq);
+    unsigned int tot_sel = all_sel ? (unsigned int)L : p;
+    const unsigned int keep_last = mode >> 8;
+    const int f0 = (kKeepLast && keep_last > 0 && !all_sel) ? max(0, L - (int)min(keep_last, (unsigned int)L)) : L;
+    if (kKeepLast && f0 < L) {
+        // the final positions the threshold leaves out, in front of this thread and in all
+        unsigned int extra = 0, left = eq_take;
+#pragma unroll
+        for (int e = 0; e < kSoloPer; ++e) {
+            if (j0 + e < L) {
+                bool keep = kr[e] > thr_key;
+                if (!keep && kr[e] == thr_key && left > 0) { keep = true; --left; }
+                extra += (!keep && j0 + e >= f0);
+            }
+        }
+        unsigned int extra_before, extra_all;
+        unsigned long long unused;
+        solo_scan(extra, 0ull, c, &extra_before, &unused, &extra_all);
+        out += extra_before;
+        tot_sel += extra_all;
+    }
+    unsigned int eq_left = eq_take;
+    unsigned long long mass = 0, all = 0;
+#pragma unroll
+    for (int e = 0; e < kSoloPer; ++e) {
+        const int j = j0 + e;
+        if (j < L) {
+            bool keep = true;
+            if (!all_sel) {
+                keep = kr[e] > thr_key;
+                if (!keep && kr[e] == thr_key && eq_left > 0) { keep = true; --eq_left; }
+                if (kKeepLast) keep = keep || (j >= f0);
+            }
+            const unsigned long long fx = to_fx(av[e]);
+            all += fx;
+            if (keep) {
+                idx[out++] = j;
+                mass += fx;
+            }
+        }
+    }
+    for (int j = tot_sel + threadIdx.x; j < L; j += kSoloThreads) idx[j] = -1;
+    if (threadIdx.x == 0) *k_out = (int32_t)tot_sel;
+    if (kept_mass) {
+        unsigned int uc;
+        unsigned long long us, kept, S_acc;
+        solo_scan(0u, mass, c, &uc, &us, nullptr, &kept);
+        solo_scan(0u, all, c, &uc, &us, nullptr, &S_acc);
+        if (threadIdx.x == 0) *kept_mass = S_acc ? (float)((double)kept / (double)S_acc) : 0.f;
+    }
+}
+
 }  // namespace
 
 size_t select_ws_bytes() { return (sizeof(GlobalHist) + 255) & ~(size_t)255; }
@@ -619,10 +1022,21 @@ size_t select_ws_bytes() { return (sizeof(GlobalHist) + 255) & ~(size_t)255; }
 zipvl_status launch_select(int L, const float *acc, const float *norm, float tau, uint32_t mode,
                            int fixed_k, int32_t *k_out, int32_t *idx, float *kept_mass, void *ws,
                            int32_t *status_word, cudaStream_t st) {
+    if (L <= kSoloMax) {
+        auto solo = (mode >> 8) ? select_solo_kernel<true> : select_solo_kernel<false>;
+        cudaError_t es = cudaFuncSetAttribute(solo, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)sizeof(SoloSmem));
+        if (es == cudaSuccess)
+            es = launch_dependent(solo, dim3(1), dim3(kSoloThreads), sizeof(SoloSmem), st, L, acc, norm, tau,
+                                  mode, fixed_k, k_out, idx, kept_mass, status_word);
+        if (es != cudaSuccess) return fail(ZIPVL_ERR_CUDA, "select: launch: %s", cudaGetErrorString(es));
+        count_launches(1);
+        return check_launch("zipvl_select");
+    }
     auto kernel = (mode >> 8) ? select_kernel<true> : select_kernel<false>;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)sizeof(SelSmem));
-    const int grid = (L <= kSoloMax) ? 1 : (L + kSelThreads - 1) / kSelThreads;
+    const int grid = (L + kSelThreads - 1) / kSelThreads;
     if (e == cudaSuccess && grid > 1) e = cudaMemsetAsync(ws, 0, sizeof(GlobalHist), st);
     if (e != cudaSuccess) return fail(ZIPVL_ERR_CUDA, "select: %s", cudaGetErrorString(e));
     e = launch_dependent(kernel, dim3(grid), dim3(kSelThreads), sizeof(SelSmem), st, L, acc, norm, tau,

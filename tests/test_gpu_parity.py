@@ -734,6 +734,33 @@ def test_prefill_layer_host_entry_point(zipvl):
     zipvl.zipvl_release_host_scratch()
 
 
+@pytest.mark.parametrize("name", ["llava7b_small_bf16", "video_gqa_small", "tiny_fp32"])
+def test_layer_step_host_entry_point_adds_a_decode_step(zipvl, name):
+    """Algorithm 1 and one step of Algorithm 2 from host buffers in one call: the prefill
+    results are those of zipvl_prefill_layer_host, the decode output is the oracle's on the
+    compacted cache with the new token appended."""
+    layer = CASES[name]()
+    Hq, Hkv, d = layer.n_q_heads, layer.n_kv_heads, layer.head_dim
+    code = {torch.bfloat16: zipvl.ZIPVL_BF16, torch.float32: zipvl.ZIPVL_F32}[layer.q.dtype]
+    desc = zipvl.zipvl_layer(layer.L, Hq, Hkv, d, code, 0, 0, 0, 0.0, 0)
+    g = torch.Generator().manual_seed(17)
+    qn = torch.randn(1, Hq, d, generator=g).to(layer.q.dtype)
+    kn = torch.randn(1, Hkv, d, generator=g).to(layer.q.dtype)
+    vn = torch.randn(1, Hkv, d, generator=g).to(layer.q.dtype)
+    k, idx, out, kc, vc, dec = zipvl.zipvl_layer_step_host(desc, layer.q, layer.k, layer.v, layer.probe_pos,
+                                                           layer.tau, qn, kn, vn)
+    k0, idx0, out0, kc0, vc0 = zipvl.zipvl_prefill_layer_host(desc, layer.q, layer.k, layer.v,
+                                                              layer.probe_pos, layer.tau)
+    assert k == k0 and torch.equal(idx, idx0) and torch.equal(out, out0)
+    assert torch.equal(kc[:k], kc0[:k]) and torch.equal(vc[:k], vc0[:k])
+    T = idx[:k].long()
+    ko = np.concatenate([to_np(layer.k[T]).reshape(-1), np.zeros(Hkv * d, np.float32)])
+    vo = np.concatenate([to_np(layer.v[T]).reshape(-1), np.zeros(Hkv * d, np.float32)])
+    seq = np.array([k], np.int32)
+    ref = oracle.decode_step(to_np(qn), to_np(kn), to_np(vn), ko, vo, np.zeros(1, np.int64), seq, Hkv)
+    check_attention(to_np(dec), ref, layer.q.dtype)
+
+
 def test_layer_step_replays_from_a_cuda_graph(zipvl):
     """score -> select -> fused prefill + compaction -> decode captured once into a CUDA
     graph (k stays on the device, nothing synchronises) and replayed on new inputs: the
