@@ -66,7 +66,7 @@ struct Barriers {
     uint64_t s_full[2];
     uint64_t p_full[2];
     uint64_t pv_done[2];
-    uint64_t tail_full[2];   // key tiles 2pt / 2pt+1 (K and V) have landed: told by the issuer
+    uint64_t tail_full[2];   // the CTA's own key tiles (K and V) have landed: told by the issuer
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -157,14 +157,21 @@ prefill_tc_kernel(LayerArgs a, const __nv_bfloat16 *__restrict__ q,
     // heaviest (longest-diagonal) pair starts first -- longest-processing-time order.
     // The grid is sized by the host's bound k_max; the pairs past the actual k map to
     // the last rows of the grid and return at once.
-    const int n_pairs = (n_valid + kPair - 1) / kPair;
+    // An odd number of 128-row tiles leaves one tile without a partner.  That single is the
+    // FIRST tile (one key tile: the cheapest item there is), and the pairs are (1,2), (3,4) ...;
+    // were the pairs counted from the front, the single would be the last tile, a CTA that
+    // walks the whole diagonal with one query tile and nothing to overlap its chain with.
+    const int n_tiles = (n_valid + kBM - 1) / kBM;
+    const int odd = n_tiles & 1;
+    const int n_pairs = (n_tiles + 1) / 2;
     const int pt = n_pairs - 1 - (int)blockIdx.y;
-    const int q0 = pt * kPair;
+    const int ta = pt > 0 ? 2 * pt - odd : 0;       // tile A of this CTA (tile B = ta + 1)
+    const int q0 = ta * kBM;
     const bool no_work = (pt < 0 || q0 >= n_valid || (int)blockIdx.x >= a.Hq);   // or a bad grid
     const int h = blockIdx.x, g = h / a.G;
-    const bool has_b = (q0 + kBM) < n_valid;        // tile B has at least one valid row
-    const int n_a = 2 * pt + 1;                     // key tiles of A (diagonal = 2pt)
-    const int n_kv = has_b ? n_a + 1 : n_a;         // key tiles of B (diagonal = 2pt+1)
+    const bool has_b = !(odd && pt == 0) && (q0 + kBM) < n_valid;   // tile B exists and has a valid row
+    const int n_a = ta + 1;                         // key tiles of A (diagonal = ta)
+    const int n_kv = has_b ? n_a + 1 : n_a;         // key tiles of B (diagonal = ta + 1)
 
     // The first token index every loading thread needs is fetched before the set-up
     // barrier, so its latency hides behind it: a softmax thread's own query row, a
@@ -250,7 +257,7 @@ prefill_tc_kernel(LayerArgs a, const __nv_bfloat16 *__restrict__ q,
                     for (int zr = r0 + sub; zr < r1; zr += 2)
                         reinterpret_cast<uint4 *>(out + ((long long)zr * a.Hq + h) * kD)[ch] = z;
                 };
-                for (int i0 = (warp - 13) * 32; i0 < kPair; i0 += 3 * 32) {
+                for (int i0 = (warp - 13) * 32; i0 < (has_b ? kPair : kBM); i0 += 3 * 32) {
                     const int i = q0 + i0 + lane;
                     const int t = token_of(i);
                     int lo = 0, hi = 0;                       // my gap: rows [lo, hi)
@@ -276,7 +283,7 @@ prefill_tc_kernel(LayerArgs a, const __nv_bfloat16 *__restrict__ q,
                 }
             }
             // Fused KV compaction (Algorithm 1: K = K[T], V = V[T]).  The last key tiles a CTA
-            // loads -- 2pt and, if tile B exists, 2pt+1 -- hold exactly the K and V rows of its
+            // loads -- its tile A and, if it has one, its tile B -- hold exactly the K and V rows of its
             // own 256 kept tokens, already gathered into shared memory for the attention.  The
             // CTA of the first query head of a KV group writes them to the compacted cache
             // from there (every (pair, kv head) once over the grid): these warps wait for the
@@ -286,11 +293,11 @@ prefill_tc_kernel(LayerArgs a, const __nv_bfloat16 *__restrict__ q,
             if (kc != nullptr && h % a.G == 0) {
                 const int lim = min(n_valid, capacity);
                 const int sub = lane >> 4, ch = lane & 15;
-                for (int j = 2 * pt; j < n_kv; ++j) {           // key tile j = kept tokens 128j ..
+                for (int j = ta; j < n_kv; ++j) {               // key tile j = kept tokens 128j ..
                     // the issuer follows the ring in order and says when K and V of this tile
                     // are in (the ring's own barriers are only meaningful to a reader that
                     // keeps up with every phase)
-                    mbar_wait(smem_u32(&bar->tail_full[j - 2 * pt]), 0, abort_flag);
+                    mbar_wait(smem_u32(&bar->tail_full[j - ta]), 0, abort_flag);
                     for (int kind = 0; kind < 2; ++kind) {       // 0: K (group 2j), 1: V (group 2j+1)
                         const int seq = 2 * j + kind;
                         const unsigned char *tile = gen + (size_t)kTileBytes * (2 + seq % kSlots);
@@ -385,8 +392,8 @@ prefill_tc_kernel(LayerArgs a, const __nv_bfloat16 *__restrict__ q,
                         // K(n+1) says that V(n) has landed too: one look at one barrier)
                         loads_ok[x] = is_full(more ? 2 * n + 2 : 2 * n + 1);
                         if (!loads_ok[x]) continue;
-                        // The last step of tile A reads key tile 2pt, that of tile B key tile
-                        // 2pt+1 -- the CTA's own 256 tokens: K and V of that tile are in now,
+                        // The last step of tile A reads the key tile of A's own tokens, that of
+                        // tile B the one of B's -- the CTA's own 256 tokens: K and V of that tile are in now,
                         // which the warps that copy them to the compacted cache are told here
                         // (once per tile: loads_ok is set once per step).
                         if (!more && leader) mbar_arrive(smem_u32(&bar->tail_full[x]));
@@ -422,7 +429,7 @@ prefill_tc_kernel(LayerArgs a, const __nv_bfloat16 *__restrict__ q,
         fence_proxy_async();
         mbar_arrive(smem_u32(&bar->q_full));
         const int n_mine = (x == 0) ? n_a : n_kv;
-        const int diag_tile = 2 * pt + x;
+        const int diag_tile = ta + x;
         if (x == 0 || has_b) {
             const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
             const uint32_t tS = lane_base + x * 128;
