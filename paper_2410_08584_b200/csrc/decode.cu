@@ -23,7 +23,6 @@ namespace zipvl {
 namespace {
 
 constexpr int kDecThreads = 128;
-constexpr int kDecUnroll = 4;
 
 __device__ __forceinline__ uint4 ld_stream(const void *p) {
     uint4 r;
@@ -54,7 +53,8 @@ __device__ __forceinline__ void unpack<float, 4>(const uint4 r, float (&x)[4]) {
     x[2] = __uint_as_float(r.z); x[3] = __uint_as_float(r.w);
 }
 
-template <typename T, int D, int GT>
+// kDecUnroll: rows per lane group in flight before any is consumed (8 where the registers allow)
+template <typename T, int D, int GT, int kDecUnroll>
 __global__ void __launch_bounds__(kDecThreads)
 decode_kernel(int Hq, int Hkv, float scale_log2, const T *__restrict__ q,
               const T *__restrict__ k_new, const T *__restrict__ v_new, T *__restrict__ k_cache,
@@ -79,6 +79,22 @@ decode_kernel(int Hq, int Hkv, float scale_log2, const T *__restrict__ q,
     const int h0 = hkv * G + qt * GT;        // first query head of this CTA
     const int n_heads = min(GT, G - qt * GT);
     const bool first = blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0;
+    // the query rows do not depend on the lengths: their loads go out together with them
+    float qv[GT][EPL];
+    {
+        const int lr_q = (threadIdx.x & 31) % LPR;
+#pragma unroll
+        for (int g = 0; g < GT; ++g) {
+            if (g < n_heads) {
+                const uint4 r = *reinterpret_cast<const uint4 *>(
+                    q + ((long long)b * Hq + h0 + g) * D + lr_q * EPL);
+                unpack<T, EPL>(r, qv[g]);
+            } else {
+#pragma unroll
+                for (int e = 0; e < EPL; ++e) qv[g][e] = 0.f;
+            }
+        }
+    }
 
     // Eq. 4: the new row goes to position seq_lens[b] if the cache has room
     // A request whose length is negative or beyond its capacity, or whose cache offset breaks
@@ -99,27 +115,19 @@ decode_kernel(int Hq, int Hkv, float scale_log2, const T *__restrict__ q,
     const int new_row = appended ? old_len : -1;
     const int c0 = blockIdx.x * chunk;
     const bool valid = c0 < len;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int rg = warp * RPW + lane / LPR;  // row group of this lane
+    const int lr = lane % LPR;               // lane inside the row
 
     if (valid) {
         const int c1 = min(len, c0 + chunk);
-        const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-        const int rg = warp * RPW + lane / LPR;  // row group of this lane
-        const int lr = lane % LPR;               // lane inside the row
-
-        float qv[GT][EPL], o[GT][EPL], m[GT], l[GT];
+        float o[GT][EPL], m[GT], l[GT];
 #pragma unroll
         for (int g = 0; g < GT; ++g) {
             m[g] = -INFINITY;
             l[g] = 0.f;
 #pragma unroll
-            for (int e = 0; e < EPL; ++e) { o[g][e] = 0.f; qv[g][e] = 0.f; }
-            if (g < n_heads) {
-                const uint4 r = *reinterpret_cast<const uint4 *>(
-                    q + ((long long)b * Hq + h0 + g) * D + lr * EPL);
-                unpack<T, EPL>(r, qv[g]);
-#pragma unroll
-                for (int e = 0; e < EPL; ++e) qv[g][e] *= scale_log2;
-            }
+            for (int e = 0; e < EPL; ++e) { o[g][e] = 0.f; qv[g][e] *= scale_log2; }
         }
 
         const long long row_pitch = (long long)Hkv * D;
@@ -219,6 +227,12 @@ decode_kernel(int Hq, int Hkv, float scale_log2, const T *__restrict__ q,
             dst[2 + c] = Os;
             if (c == 0) { dst[0] = M; dst[1] = Ls; }
         }
+    } else if ((int)threadIdx.x < n_heads) {
+        // a chunk past the request's length: an empty partial (the merge reads every chunk slot
+        // without waiting for the length)
+        float *dst = ws + (((long long)b * Hq + h0 + threadIdx.x) * n_chunks + blockIdx.x) * (D + 2);
+        dst[0] = -INFINITY;
+        dst[1] = 0.f;
     }
 
     // the length this step attends over, for the merge kernel (which must not read
@@ -230,9 +244,13 @@ decode_kernel(int Hq, int Hkv, float scale_log2, const T *__restrict__ q,
 }
 
 // Second kernel of a step: merges the per-chunk partial results of one request's query
-// heads (online softmax merge in chunk order), writes the output, and bumps the
-// request's length.  Launched as a programmatic dependent of the kernel above, so it is
-// staged while that one runs; no tickets, no counters to clear.
+// heads (online-softmax merge), writes the output, and bumps the request's length.
+// Launched as a programmatic dependent of the kernel above, so it is staged while that one
+// runs; no tickets, no counters to clear.  Eight adjacent lanes share one (head, channel):
+// lane p takes chunks p, p + 8, ... -- every chunk slot holds a partial, an empty one past the
+// request's length, so all loads go out at once without waiting for the length -- and the
+// eight are merged by shuffles in a fixed order.
+constexpr int kMergeLanes = 8;
 template <typename T, int D>
 __global__ void __launch_bounds__(256)
 decode_merge_kernel(int Hq, int chunk, int n_chunks, const float *__restrict__ ws,
@@ -240,40 +258,52 @@ decode_merge_kernel(int Hq, int chunk, int n_chunks, const float *__restrict__ w
     grid_launch_dependents();
     grid_dependency_wait(ws, lens, seq_lens);
     const int b = blockIdx.y;
-    const int len = lens[2 * b];
-    const int n_valid_chunks = (len + chunk - 1) / chunk;
-    const int t = blockIdx.x * 256 + threadIdx.x;       // (head, channel) of this thread
-    if (t < Hq * D) {
-        const int hq = t / D, c = t % D;
-        const float *src = ws + ((long long)b * Hq + hq) * n_chunks * (D + 2);
-        // one pass, eight chunks (24 loads) in flight, merged online in chunk order
-        float M = -INFINITY, Ls = 0.f, Os = 0.f;
-        for (int i0 = 0; i0 < n_valid_chunks; i0 += 8) {
-            float mi[8], li[8], oi[8];
+    const int t = (blockIdx.x * 256 + threadIdx.x) / kMergeLanes;       // (head, channel) of this lane group
+    const int part = threadIdx.x % kMergeLanes;
+    const bool live = t < Hq * D;
+    const int hq = live ? t / D : 0, c = live ? t % D : 0;
+    const float *src = ws + ((long long)b * Hq + hq) * n_chunks * (D + 2);
+    float M = -INFINITY, Ls = 0.f, Os = 0.f;
+    for (int i0 = part; i0 < n_chunks; i0 += 8 * kMergeLanes) {
+        float mi[8], li[8], oi[8];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                const bool in = i0 + u < n_valid_chunks;
-                const float *p = src + (long long)(in ? i0 + u : i0) * (D + 2);
-                mi[u] = in ? __ldcg(p) : -INFINITY;
-                li[u] = __ldcg(p + 1);
-                oi[u] = __ldcg(p + 2 + c);
-            }
+        for (int u = 0; u < 8; ++u) {
+            const int i = i0 + u * kMergeLanes;
+            const bool in = live && i < n_chunks;
+            const float *p = src + (long long)(in ? i : 0) * (D + 2);
+            mi[u] = in ? __ldcg(p) : -INFINITY;
+            li[u] = in ? __ldcg(p + 1) : 0.f;
+            oi[u] = in ? __ldcg(p + 2 + c) : 0.f;
+        }
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                if (mi[u] != -INFINITY) {
-                    const float Mn = fmaxf(M, mi[u]);
-                    const float wo = fast_exp2(M - Mn), wn = fast_exp2(mi[u] - Mn);
-                    Ls = Ls * wo + li[u] * wn;
-                    Os = Os * wo + oi[u] * wn;
-                    M = Mn;
-                }
+        for (int u = 0; u < 8; ++u) {
+            if (mi[u] != -INFINITY) {
+                const float Mn = fmaxf(M, mi[u]);
+                const float wo = fast_exp2(M - Mn), wn = fast_exp2(mi[u] - Mn);
+                Ls = Ls * wo + li[u] * wn;
+                Os = Os * wo + oi[u] * wn;
+                M = Mn;
             }
         }
-        // (an empty cache with nothing appended has no chunks: the output is zero)
-        store_elem(out + ((long long)b * Hq + hq) * D + c, Ls > 0.f ? Os / Ls : 0.f);
     }
+#pragma unroll
+    for (int o = 1; o < kMergeLanes; o <<= 1) {
+        const float M2 = __shfl_xor_sync(0xffffffffu, M, o);
+        const float L2 = __shfl_xor_sync(0xffffffffu, Ls, o);
+        const float O2 = __shfl_xor_sync(0xffffffffu, Os, o);
+        const float Mn = fmaxf(M, M2);
+        // (the two sides of a pair compute the same sum in the same order of operands)
+        const float w1 = (M == -INFINITY) ? 0.f : fast_exp2(M - Mn);
+        const float w2 = (M2 == -INFINITY) ? 0.f : fast_exp2(M2 - Mn);
+        const bool lo = (part & o) == 0;
+        Ls = lo ? (Ls * w1 + L2 * w2) : (L2 * w2 + Ls * w1);
+        Os = lo ? (Os * w1 + O2 * w2) : (O2 * w2 + Os * w1);
+        M = Mn;
+    }
+    // (an empty cache with nothing appended has only empty partials: the output is zero)
+    if (live && part == 0) store_elem(out + ((long long)b * Hq + hq) * D + c, Ls > 0.f ? Os / Ls : 0.f);
     // Eq. 4: the appended row now counts
-    if (blockIdx.x == 0 && threadIdx.x == 0 && lens[2 * b + 1]) seq_lens[b] = len;
+    if (blockIdx.x == 0 && threadIdx.x == 0 && lens[2 * b + 1]) seq_lens[b] = lens[2 * b];
 }
 
 // Cache rows per CTA: small problems get small chunks so that every SM still has
@@ -305,7 +335,7 @@ zipvl_status run(const zipvl_decode_desc &d, float scale_log2, const void *q, co
 #define ZIPVL_DEC(GT_)                                                                          \
     {                                                                                           \
         dim3 grid(n_chunks, Hkv * ((G + GT_ - 1) / GT_), B);                                    \
-        le = launch_dependent(decode_kernel<T, D, GT_>, grid, dim3(kDecThreads), 0, st, Hq, Hkv,     \
+        le = launch_dependent(decode_kernel<T, D, GT_, (GT_ <= 2 ? 8 : 4)>, grid, dim3(kDecThreads), 0, st, Hq, Hkv, \
                               scale_log2, (const T *)q, (const T *)k_new, (const T *)v_new,           \
                               (T *)k_cache, (T *)v_cache, cache_off, capacity, seq_lens, max_len,    \
                               chunk, n_chunks, wsf, lens, (T *)out, status_word);                    \
@@ -317,7 +347,7 @@ zipvl_status run(const zipvl_decode_desc &d, float scale_log2, const void *q, co
     else ZIPVL_DEC(8)
 #undef ZIPVL_DEC
     if (le == cudaSuccess)
-        le = launch_dependent(decode_merge_kernel<T, D>, dim3((Hq * D + 255) / 256, B), dim3(256), 0, st, Hq,
+        le = launch_dependent(decode_merge_kernel<T, D>, dim3((Hq * D * kMergeLanes + 255) / 256, B), dim3(256), 0, st, Hq,
                               chunk, n_chunks, (const float *)wsf, (const int *)lens, seq_lens, (T *)out);
     if (le != cudaSuccess) return fail(ZIPVL_ERR_CUDA, "zipvl_decode: launch: %s", cudaGetErrorString(le));
     count_launches(2);
