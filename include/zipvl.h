@@ -258,6 +258,27 @@ zipvl_status zipvl_decode(const zipvl_decode_desc *desc, const void *q, const vo
                           int32_t *status_word, void *stream);
 
 /*
+ * zipvl_decode_paged -- zipvl_decode over a paged cache.
+ * Paper: Algorithm 2, Eq. 4-5, as zipvl_decode; only the storage of the kept cache differs
+ * (serving systems keep caches that grow token by token in fixed-size pages of a shared pool).
+ *
+ *   k_pages, v_pages: device pools [n_pages, page_rows, Hkv, d]; page_rows a power of two
+ *   from 16 to 1024.  block_table: device int32 [batch, table_stride]; request b's row r is
+ *   row r % page_rows of page block_table[b * table_stride + r / page_rows].
+ *   capacity[b]: rows request b may hold (its pages x page_rows); table_stride must cover
+ *   max_len rows.  Everything else as zipvl_decode (append at row seq_lens[b], attention over
+ *   all rows, ZIPVL_DEV_CAPACITY for a full cache).  A page number outside [0, n_pages) is
+ *   reported as ZIPVL_DEV_BAD_INDEX and its rows are left out of the attention.
+ * ws: zipvl_workspace_bytes(ZIPVL_OP_DECODE) as for zipvl_decode.
+ */
+zipvl_status zipvl_decode_paged(const zipvl_decode_desc *desc, const void *q, const void *k_new,
+                                const void *v_new, void *k_pages, void *v_pages,
+                                const int32_t *block_table, int32_t table_stride,
+                                int32_t page_rows, int32_t n_pages, const int32_t *capacity,
+                                int32_t *seq_lens, int32_t max_len, void *out, void *ws,
+                                size_t ws_bytes, int32_t *status_word, void *stream);
+
+/*
  * zipvl_decode_noalloc -- zipvl_decode for callers that cannot allocate.
  * (The paper has no counterpart: this is a deployment variant of the decode
  * step, same arithmetic, same kernels.)

@@ -198,3 +198,36 @@ def decode_step(q, k_new, v_new, k_cache, v_cache, cache_off, seq_lens, n_kv_hea
                     B, Hq, int(n_kv_heads), d,
                     default_scale(d) if scale is None else float(scale), out)
     return out
+
+
+def decode_step_paged(q, k_new, v_new, k_pages, v_pages, block_table, seq_lens, scale=None):
+    """Algorithm 2 (Eq. 4-5) where each request's cache is a list of pages of a shared pool: a
+    storage layout, not a change of the method.  k_pages / v_pages are float32
+    [n_pages, page_rows, Hkv, d] updated in place; block_table int32 [B, max_pages] names, in
+    order, the pages that hold request b's rows.  Each request's rows are gathered into a
+    contiguous cache, decode_step runs on those, and the appended rows are written back to the
+    page they belong to.  Returns float64 [B, Hq, d]."""
+    q = _f32(q)
+    B = q.shape[0]
+    n_pages, page_rows, Hkv, d = k_pages.shape
+    block_table = np.asarray(block_table, np.int64)
+    row = Hkv * d
+    cap = block_table.shape[1] * page_rows
+    kc = np.zeros((B, cap, Hkv, d), np.float32)
+    vc = np.zeros_like(kc)
+    for b in range(B):
+        n_used = -(-(int(seq_lens[b]) + 1) // page_rows)          # pages that hold rows, with room for one more
+        for i in range(min(n_used, block_table.shape[1])):
+            kc[b, i * page_rows:(i + 1) * page_rows] = k_pages[block_table[b, i]]
+            vc[b, i * page_rows:(i + 1) * page_rows] = v_pages[block_table[b, i]]
+    off = (np.arange(B, dtype=np.int64) * cap * row)
+    old = np.array(seq_lens, np.int32).copy()
+    out = decode_step(q, k_new, v_new, kc.reshape(-1), vc.reshape(-1), off, seq_lens, Hkv, scale)
+    if k_new is not None:
+        for b in range(B):
+            r = int(old[b])
+            if int(seq_lens[b]) == r + 1:                          # the row was appended
+                page = block_table[b, r // page_rows]
+                k_pages[page, r % page_rows] = kc[b, r]
+                v_pages[page, r % page_rows] = vc[b, r]
+    return out

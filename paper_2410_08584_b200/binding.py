@@ -25,7 +25,7 @@ EXPORTS = ["zipvl_status_string", "zipvl_last_error", "zipvl_version", "zipvl_la
            "zipvl_workspace_bytes",
            "zipvl_score", "zipvl_select", "zipvl_sparse_prefill", "zipvl_compact_kv",
            "zipvl_sparse_prefill_compact",
-           "zipvl_decode", "zipvl_decode_noalloc", "zipvl_prefill_layer_host", "zipvl_layer_step_host",
+           "zipvl_decode", "zipvl_decode_paged", "zipvl_decode_noalloc", "zipvl_prefill_layer_host", "zipvl_layer_step_host",
            "zipvl_release_host_scratch", "zipvl_selftest_wait_timeout"]
 
 
@@ -84,6 +84,9 @@ def load():
     lib.zipvl_decode.restype = C.c_int
     lib.zipvl_decode.argtypes = [C.POINTER(zipvl_decode_desc), vp, vp, vp, vp, vp, vp, vp, vp,
                                  i32, vp, vp, sz, vp, vp]
+    lib.zipvl_decode_paged.restype = C.c_int
+    lib.zipvl_decode_paged.argtypes = [C.POINTER(zipvl_decode_desc), vp, vp, vp, vp, vp, vp, i32, i32, i32,
+                                       vp, vp, i32, vp, vp, sz, vp, vp]
     lib.zipvl_decode_noalloc.restype = C.c_int
     lib.zipvl_decode_noalloc.argtypes = [C.POINTER(zipvl_decode_desc), vp, vp, vp, vp, vp, vp, vp,
                                          vp, i32, vp, vp, vp]
@@ -270,6 +273,26 @@ def zipvl_decode(desc, q, k_new, v_new, k_cache, v_cache, cache_off, capacity, s
                                _ptr(v_cache), _ptr(cache_off), _ptr(capacity), _ptr(seq_lens),
                                int(max_len), _ptr(out), _ptr(ws), ws.numel(), _ptr(status),
                                _stream(stream)))
+    return out
+
+
+def zipvl_decode_paged(desc, q, k_new, v_new, k_pages, v_pages, block_table, capacity, seq_lens, max_len,
+                       out=None, ws=None, status=None, stream=None):
+    """One decode step over paged caches: k_pages / v_pages [n_pages, page_rows, Hkv, d],
+    block_table int32 [B, max_pages]; returns out [B,Hq,d]."""
+    _dev(q, "q"), _dev(k_pages, "k_pages"), _dev(v_pages, "v_pages")
+    _dev(block_table, "block_table", torch.int32), _dev(capacity, "capacity", torch.int32)
+    _dev(seq_lens, "seq_lens", torch.int32)
+    out = torch.empty_like(q) if out is None else out
+    if ws is None:
+        lay = zipvl_layer(int(max_len), desc.n_q_heads, desc.n_kv_heads, desc.head_dim, desc.dtype,
+                          0, 0, 0, 0.0, 0)
+        ws = workspace(zipvl_workspace_bytes(OP_DECODE, lay, 0, desc.batch), q.device)
+    _check(load().zipvl_decode_paged(C.byref(desc), _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(k_pages),
+                                     _ptr(v_pages), _ptr(block_table), block_table.shape[1],
+                                     k_pages.shape[1], k_pages.shape[0], _ptr(capacity), _ptr(seq_lens),
+                                     int(max_len), _ptr(out), _ptr(ws), ws.numel(), _ptr(status),
+                                     _stream(stream)))
     return out
 
 

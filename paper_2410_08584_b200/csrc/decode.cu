@@ -24,6 +24,13 @@ namespace {
 
 constexpr int kDecThreads = 128;
 
+// Paged cache: request b's row r lives in page table[b * stride + (r >> shift)] of a pool of
+// n_pages pages of (1 << shift) rows each.  table == nullptr: contiguous caches at cache_off.
+struct PageArgs {
+    const int32_t *table;
+    int stride, shift, n_pages;
+};
+
 __device__ __forceinline__ uint4 ld_stream(const void *p) {
     uint4 r;
     asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
@@ -58,7 +65,7 @@ template <typename T, int D, int GT, int kDecUnroll>
 __global__ void __launch_bounds__(kDecThreads)
 decode_kernel(int Hq, int Hkv, float scale_log2, const T *__restrict__ q,
               const T *__restrict__ k_new, const T *__restrict__ v_new, T *__restrict__ k_cache,
-              T *__restrict__ v_cache, const int64_t *__restrict__ cache_off,
+              T *__restrict__ v_cache, const int64_t *__restrict__ cache_off, PageArgs pg,
               const int32_t *__restrict__ capacity, int32_t *__restrict__ seq_lens, int max_len,
               int chunk, int n_chunks, float *__restrict__ ws, int *__restrict__ lens,
               T *__restrict__ out, int32_t *status_word) {
@@ -71,7 +78,7 @@ decode_kernel(int Hq, int Hkv, float scale_log2, const T *__restrict__ q,
 
     grid_launch_dependents();
     // lengths and caches may be the previous kernel's output
-    grid_dependency_wait(q, k_new, v_new, k_cache, v_cache, cache_off, capacity, seq_lens);
+    grid_dependency_wait(q, k_new, v_new, k_cache, v_cache, cache_off, capacity, seq_lens, pg.table);
     const int G = Hq / Hkv;
     const int q_tiles = (G + GT - 1) / GT;
     const int hkv = blockIdx.y / q_tiles, qt = blockIdx.y % q_tiles;
@@ -102,8 +109,8 @@ decode_kernel(int Hq, int Hkv, float scale_log2, const T *__restrict__ q,
     // zero output) and reported: none of its rows can be trusted to lie inside the cache.
     const int old_len = seq_lens[b];
     const int cap = capacity[b];
-    const bool bad = old_len < 0 || old_len > cap ||
-                     ((cache_off[b] * (long long)sizeof(T)) & 15) != 0;
+    const long long coff = pg.table ? 0ll : cache_off[b];
+    const bool bad = old_len < 0 || old_len > cap || ((coff * (long long)sizeof(T)) & 15) != 0;
     if (bad && first) report(status_word, ZIPVL_DEV_BAD_INDEX);
     const bool appended = !bad && k_new != nullptr && old_len < cap;
     if (k_new != nullptr && !bad && !appended && first) report(status_word, ZIPVL_DEV_CAPACITY);
@@ -132,8 +139,17 @@ decode_kernel(int Hq, int Hkv, float scale_log2, const T *__restrict__ q,
 
         const long long row_pitch = (long long)Hkv * D;
         const long long head_off = (long long)hkv * D + lr * EPL;
-        T *kb = k_cache + cache_off[b] + head_off;
-        T *vb = v_cache + cache_off[b] + head_off;
+        T *kb = k_cache + coff + head_off;
+        T *vb = v_cache + coff + head_off;
+        // element offset of a cache row from kb / vb; -1 for a page outside the pool (reported,
+        // the row is skipped)
+        const int32_t *my_table = pg.table ? pg.table + (long long)b * pg.stride : nullptr;
+        auto row_off = [&](int row) -> long long {
+            if (my_table == nullptr) return row * row_pitch;
+            const int page = my_table[row >> pg.shift];
+            if (page < 0 || page >= pg.n_pages) { report(status_word, ZIPVL_DEV_BAD_INDEX); return -1; }
+            return (((long long)page << pg.shift) + (row & ((1 << pg.shift) - 1))) * row_pitch;
+        };
 
         for (int base = c0; base < c1; base += NG * kDecUnroll) {
             uint4 kk[kDecUnroll], vv[kDecUnroll];
@@ -142,16 +158,18 @@ decode_kernel(int Hq, int Hkv, float scale_log2, const T *__restrict__ q,
             for (int u = 0; u < kDecUnroll; ++u) {
                 const int row = base + u * NG + rg;
                 ok[u] = row < c1;
+                const long long ro = ok[u] ? row_off(row) : -1;
+                ok[u] = ok[u] && ro >= 0;
                 if (ok[u] && row != new_row) {
-                    kk[u] = ld_stream(kb + row * row_pitch);
-                    vv[u] = ld_stream(vb + row * row_pitch);
+                    kk[u] = ld_stream(kb + ro);
+                    vv[u] = ld_stream(vb + ro);
                 } else if (ok[u]) {
                     // the appended token: read it from k_new / v_new, store it on the way
                     kk[u] = *reinterpret_cast<const uint4 *>(k_new + (long long)b * row_pitch + head_off);
                     vv[u] = *reinterpret_cast<const uint4 *>(v_new + (long long)b * row_pitch + head_off);
                     if (qt == 0) {
-                        *reinterpret_cast<uint4 *>(kb + row * row_pitch) = kk[u];
-                        *reinterpret_cast<uint4 *>(vb + row * row_pitch) = vv[u];
+                        *reinterpret_cast<uint4 *>(kb + ro) = kk[u];
+                        *reinterpret_cast<uint4 *>(vb + ro) = vv[u];
                     }
                 } else {
                     kk[u] = make_uint4(0, 0, 0, 0);
@@ -324,7 +342,7 @@ size_t counter_bytes(int B, int) { return (size_t)(2 * B) * sizeof(int); }   // 
 
 template <typename T, int D>
 zipvl_status run(const zipvl_decode_desc &d, float scale_log2, const void *q, const void *k_new,
-                 const void *v_new, void *k_cache, void *v_cache, const int64_t *cache_off,
+                 const void *v_new, void *k_cache, void *v_cache, const int64_t *cache_off, PageArgs pg,
                  const int32_t *capacity, int32_t *seq_lens, int max_len, void *out, void *ws,
                  int32_t *status_word, cudaStream_t st) {
     const int B = d.batch, Hq = d.n_q_heads, Hkv = d.n_kv_heads, G = Hq / Hkv;
@@ -337,7 +355,7 @@ zipvl_status run(const zipvl_decode_desc &d, float scale_log2, const void *q, co
         dim3 grid(n_chunks, Hkv * ((G + GT_ - 1) / GT_), B);                                    \
         le = launch_dependent(decode_kernel<T, D, GT_, (GT_ <= 2 ? 8 : 4)>, grid, dim3(kDecThreads), 0, st, Hq, Hkv, \
                               scale_log2, (const T *)q, (const T *)k_new, (const T *)v_new,           \
-                              (T *)k_cache, (T *)v_cache, cache_off, capacity, seq_lens, max_len,    \
+                              (T *)k_cache, (T *)v_cache, cache_off, pg, capacity, seq_lens, max_len, \
                               chunk, n_chunks, wsf, lens, (T *)out, status_word);                    \
     }
     cudaError_t le = cudaSuccess;
@@ -360,12 +378,13 @@ size_t decode_ws_bytes(int B, int Hq, int D, int max_len) {
     return partial_bytes(B, Hq, D, max_len) + counter_bytes(B, Hq);
 }
 
-zipvl_status launch_decode(const zipvl_decode_desc &d, float scale_log2, const void *q,
-                           const void *k_new, const void *v_new, void *k_cache, void *v_cache,
-                           const int64_t *cache_off, const int32_t *capacity, int32_t *seq_lens,
-                           int max_len, void *out, void *ws, int32_t *status_word,
-                           cudaStream_t st) {
-#define ZIPVL_ARGS d, scale_log2, q, k_new, v_new, k_cache, v_cache, cache_off, capacity, \
+namespace {
+zipvl_status dispatch_decode(const zipvl_decode_desc &d, float scale_log2, const void *q,
+                             const void *k_new, const void *v_new, void *k_cache, void *v_cache,
+                             const int64_t *cache_off, PageArgs pg, const int32_t *capacity,
+                             int32_t *seq_lens, int max_len, void *out, void *ws,
+                             int32_t *status_word, cudaStream_t st) {
+#define ZIPVL_ARGS d, scale_log2, q, k_new, v_new, k_cache, v_cache, cache_off, pg, capacity, \
                    seq_lens, max_len, out, ws, status_word, st
     if (d.dtype == ZIPVL_BF16) {
         if (d.head_dim == 128) return run<__nv_bfloat16, 128>(ZIPVL_ARGS);
@@ -379,6 +398,16 @@ zipvl_status launch_decode(const zipvl_decode_desc &d, float scale_log2, const v
     }
 #undef ZIPVL_ARGS
     return fail(ZIPVL_ERR_UNSUPPORTED, "decode: head_dim %d", d.head_dim);
+}
+}  // namespace
+
+zipvl_status launch_decode(const zipvl_decode_desc &d, float scale_log2, const void *q,
+                           const void *k_new, const void *v_new, void *k_cache, void *v_cache,
+                           const int64_t *cache_off, const int32_t *capacity, int32_t *seq_lens,
+                           int max_len, void *out, void *ws, int32_t *status_word,
+                           cudaStream_t st) {
+    return dispatch_decode(d, scale_log2, q, k_new, v_new, k_cache, v_cache, cache_off,
+                           PageArgs{nullptr, 0, 0, 0}, capacity, seq_lens, max_len, out, ws, status_word, st);
 }
 
 // ---- decode without any allocation ------------------------------------------
@@ -453,4 +482,48 @@ extern "C" zipvl_status zipvl_decode_noalloc(const zipvl_decode_desc *d, const v
     const float scale = d->softmax_scale > 0.f ? d->softmax_scale : 1.0f / sqrtf((float)d->head_dim);
     return launch_decode(*d, scale * kLog2e, q, k_new, v_new, k_cache, v_cache, cache_off, capacity,
                          seq_lens, max_len, out, scratch, status_word, (cudaStream_t)stream);
+}
+
+
+// ---- decode over a paged cache -------------------------------------------------
+extern "C" zipvl_status zipvl_decode_paged(const zipvl_decode_desc *d, const void *q,
+                                           const void *k_new, const void *v_new, void *k_pages,
+                                           void *v_pages, const int32_t *block_table,
+                                           int32_t table_stride, int32_t page_rows, int32_t n_pages,
+                                           const int32_t *capacity, int32_t *seq_lens,
+                                           int32_t max_len, void *out, void *ws, size_t ws_bytes,
+                                           int32_t *status_word, void *stream) {
+    using namespace zipvl;
+    const char *who = "zipvl_decode_paged";
+    if (!d) return fail(ZIPVL_ERR_INVALID_ARG, "%s: desc is NULL", who);
+    if (d->batch < 1 || d->batch > 65535 || d->n_q_heads < 1 || d->n_kv_heads < 1 ||
+        d->n_q_heads % d->n_kv_heads)
+        return fail(ZIPVL_ERR_INVALID_ARG, "%s: batch %d heads %d / %d", who, d->batch,
+                    d->n_q_heads, d->n_kv_heads);
+    if ((d->dtype != ZIPVL_BF16 && d->dtype != ZIPVL_F32 && d->dtype != ZIPVL_F16) ||
+        (d->head_dim != 64 && d->head_dim != 128) || d->n_q_heads / d->n_kv_heads > 8)
+        return fail(ZIPVL_ERR_UNSUPPORTED, "%s: dtype %d head_dim %d group %d", who, d->dtype,
+                    d->head_dim, d->n_q_heads / d->n_kv_heads);
+    if (!q || !k_pages || !v_pages || !block_table || !capacity || !seq_lens || !out || !ws)
+        return fail(ZIPVL_ERR_INVALID_ARG, "%s: NULL pointer", who);
+    if ((k_new == NULL) != (v_new == NULL))
+        return fail(ZIPVL_ERR_INVALID_ARG, "%s: k_new and v_new must both be given or both NULL", who);
+    if (max_len < 1) return fail(ZIPVL_ERR_INVALID_ARG, "%s: max_len = %d", who, max_len);
+    int shift = 0;
+    while ((1 << shift) < page_rows) ++shift;
+    if (page_rows < 16 || page_rows > 1024 || (1 << shift) != page_rows)
+        return fail(ZIPVL_ERR_INVALID_ARG, "%s: page_rows = %d (a power of two from 16 to 1024)", who, page_rows);
+    if (n_pages < 1 || table_stride < (max_len + page_rows - 1) / page_rows)
+        return fail(ZIPVL_ERR_INVALID_ARG, "%s: n_pages = %d, table_stride = %d for max_len %d", who,
+                    n_pages, table_stride, max_len);
+    if (!(d->softmax_scale >= 0.f) || isinf(d->softmax_scale))
+        return fail(ZIPVL_ERR_INVALID_ARG, "%s: softmax_scale", who);
+    if (((uintptr_t)q | (uintptr_t)k_pages | (uintptr_t)v_pages | (uintptr_t)out | (uintptr_t)ws) & 15u)
+        return fail(ZIPVL_ERR_INVALID_ARG, "%s: tensors must be 16-byte aligned", who);
+    const size_t need = (decode_ws_bytes(d->batch, d->n_q_heads, d->head_dim, max_len) + 255) & ~(size_t)255;
+    if (ws_bytes < need) return fail(ZIPVL_ERR_WORKSPACE, "%s: workspace %zu < %zu", who, ws_bytes, need);
+    const float scale = d->softmax_scale > 0.f ? d->softmax_scale : 1.0f / sqrtf((float)d->head_dim);
+    return dispatch_decode(*d, scale * kLog2e, q, k_new, v_new, k_pages, v_pages, nullptr,
+                           PageArgs{block_table, table_stride, shift, n_pages}, capacity, seq_lens,
+                           max_len, out, ws, status_word, (cudaStream_t)stream);
 }

@@ -687,6 +687,58 @@ def test_decode_parity(zipvl, lens, Hq, Hkv, d, dtype):
     assert st.item() & zipvl.DEV_CAPACITY and np.array_equal(seq_d.cpu().numpy(), seq_o)
 
 
+@pytest.mark.parametrize("lens,Hq,Hkv,d,dtype,page_rows", [
+    ([700, 1, 300, 1025, 17, 0], 8, 8, 128, torch.bfloat16, 64),
+    ([513, 40, 2000], 14, 2, 128, torch.bfloat16, 128),
+    ([100, 259, 64], 4, 1, 64, torch.float16, 16),
+    ([300, 7], 4, 4, 64, torch.float32, 64),
+])
+def test_paged_decode_parity(zipvl, lens, Hq, Hkv, d, dtype, page_rows):
+    """Decode over caches scattered in pages of a shared pool (shuffled page numbers), three
+    steps with appends that cross page boundaries, against the oracle's paged decode."""
+    B, steps = len(lens), 3
+    g = torch.Generator().manual_seed(sum(lens) + page_rows)
+    pages_per = [-(-(n + steps) // page_rows) for n in lens]
+    max_pages = max(pages_per)
+    n_pages = sum(pages_per) + 3
+    perm = torch.randperm(n_pages, generator=g)
+    table = torch.full((B, max_pages), -1, dtype=torch.int32)
+    pos = 0
+    for b in range(B):
+        table[b, :pages_per[b]] = perm[pos:pos + pages_per[b]].to(torch.int32)
+        pos += pages_per[b]
+    k_pages = torch.randn(n_pages, page_rows, Hkv, d, generator=g).to(dtype)
+    v_pages = torch.randn(n_pages, page_rows, Hkv, d, generator=g).to(dtype)
+    cap = torch.tensor([p_ * page_rows for p_ in pages_per], dtype=torch.int32)
+    code = {torch.bfloat16: zipvl.ZIPVL_BF16, torch.float32: zipvl.ZIPVL_F32, torch.float16: zipvl.ZIPVL_F16}[dtype]
+    desc = zipvl.zipvl_decode_desc(B, Hq, Hkv, d, code, 0.0)
+    kp_d, vp_d, table_d, cap_d = k_pages.to(DEV), v_pages.to(DEV), table.to(DEV), cap.to(DEV)
+    seq_d = torch.tensor(lens, dtype=torch.int32, device=DEV)
+    kp_o, vp_o = k_pages.float().numpy().copy(), v_pages.float().numpy().copy()
+    table_o = table.clamp(min=0).numpy()            # the oracle never touches the unused entries
+    seq_o = np.array(lens, np.int32)
+    st = status_word()
+    max_len = max(lens) + steps
+    for step in range(steps):
+        q = torch.randn(B, Hq, d, generator=g).to(dtype)
+        kn = torch.randn(B, Hkv, d, generator=g).to(dtype)
+        vn = torch.randn(B, Hkv, d, generator=g).to(dtype)
+        out = zipvl.zipvl_decode_paged(desc, q.to(DEV), kn.to(DEV), vn.to(DEV), kp_d, vp_d, table_d, cap_d,
+                                       seq_d, max_len, status=st)
+        ref = oracle.decode_step_paged(to_np(q), to_np(kn), to_np(vn), kp_o, vp_o, table_o, seq_o)
+        check_attention(to_np(out), ref, dtype)
+        assert np.array_equal(seq_d.cpu().numpy(), seq_o)
+    assert st.item() == 0
+    # the pools after the appends are identical (appended rows are copied bit for bit)
+    assert np.array_equal(kp_d.float().cpu().numpy(), kp_o) and np.array_equal(vp_d.float().cpu().numpy(), vp_o)
+    # a page number outside the pool: reported, the rows of that page left out, nothing faults
+    bad = table_d.clone()
+    bad[0, 0] = n_pages + 5
+    zipvl.zipvl_decode_paged(desc, q.to(DEV), None, None, kp_d, vp_d, bad, cap_d, seq_d, max_len, status=st)
+    torch.cuda.synchronize()
+    assert st.item() & zipvl.DEV_BAD_INDEX
+
+
 def test_decode_on_compacted_cache_matches_oracle_pipeline(zipvl):
     """prefill -> compaction -> decode chained on the device without host sync of k."""
     layer = CASES["llava7b_small_bf16"]()

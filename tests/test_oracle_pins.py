@@ -466,3 +466,37 @@ def test_worked_example_end_to_end():
                            np.zeros(1, np.int64), seq, 1, scale=scale)
     np.testing.assert_allclose(o.ravel(), [float(g["decode_out"][0])], rtol=1e-14)
     assert seq[0] == 3
+
+
+def test_paged_decode_is_decode_on_the_gathered_rows():
+    """The paged layout is storage only: with any permutation of the pool's pages the outputs
+    equal those of decode_step on contiguous caches holding the same rows, the appended row
+    lands in the page and slot its position names, and no other pool entry changes."""
+    rng = np.random.default_rng(12)
+    B, Hq, Hkv, d, page_rows = 3, 4, 2, 8, 4
+    lens = np.array([7, 4, 0], np.int32)            # mid-page, page boundary (append opens a new page), empty
+    max_pages = 3
+    n_pages = 11
+    perm = rng.permutation(n_pages)[: B * max_pages].reshape(B, max_pages).astype(np.int32)
+    k_pages = rng.standard_normal((n_pages, page_rows, Hkv, d)).astype(np.float32)
+    v_pages = rng.standard_normal((n_pages, page_rows, Hkv, d)).astype(np.float32)
+    q = rng.standard_normal((B, Hq, d)).astype(np.float32)
+    kn = rng.standard_normal((B, Hkv, d)).astype(np.float32)
+    vn = rng.standard_normal((B, Hkv, d)).astype(np.float32)
+    # contiguous reference built by hand from the table
+    cap = max_pages * page_rows
+    kc = np.stack([np.concatenate([k_pages[p_] for p_ in perm[b]]) for b in range(B)])
+    vc = np.stack([np.concatenate([v_pages[p_] for p_ in perm[b]]) for b in range(B)])
+    off = np.arange(B, dtype=np.int64) * cap * Hkv * d
+    seq_ref = lens.copy()
+    kc_flat, vc_flat = kc.reshape(-1).copy(), vc.reshape(-1).copy()
+    want = oracle.decode_step(q, kn, vn, kc_flat, vc_flat, off, seq_ref, Hkv)
+    kp, vp, seq = k_pages.copy(), v_pages.copy(), lens.copy()
+    got = oracle.decode_step_paged(q, kn, vn, kp, vp, perm, seq)
+    assert np.array_equal(got, want) and np.array_equal(seq, lens + 1)
+    changed = np.argwhere((kp != k_pages).any(axis=(2, 3)))
+    expect = sorted((int(perm[b, lens[b] // page_rows]), int(lens[b] % page_rows)) for b in range(B))
+    assert sorted(map(tuple, changed.tolist())) == expect
+    for b in range(B):
+        assert np.array_equal(kp[perm[b, lens[b] // page_rows], lens[b] % page_rows], kn[b])
+        assert np.array_equal(vp[perm[b, lens[b] // page_rows], lens[b] % page_rows], vn[b])
