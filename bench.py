@@ -450,6 +450,60 @@ def stack_benchmark(z, dev, n_layers, peaks, reps=5):
             "note": "score, select, sparse prefill + compaction (one call) per layer, whole stack on one stream"}
 
 
+def batched_benchmark(z, dev, layers, peaks, n_seq=4, reps=40):
+    """Several sequences of the benchmark's shape per call (zipvl_score_batch, zipvl_select_batch,
+    zipvl_sparse_prefill_batch with compaction): one launch per kernel for the whole batch.  Two
+    batches alternate (each 4 x 72 MB, so nothing is served from L2 across calls)."""
+    batches = []
+    for lo in (0, len(layers) - n_seq):
+        ls = layers[lo:lo + n_seq]
+        batches.append(tuple(torch.stack([getattr(l, a) for l in ls]).to(dev) for a in ("q", "k", "v")) +
+                       (torch.stack([l.probe_pos for l in ls]).to(dev),))
+    L, Hq, d = layers[0].L, layers[0].n_q_heads, layers[0].head_dim
+    Hkv = layers[0].n_kv_heads
+    acc = torch.empty(n_seq, L, dtype=torch.float32, device=dev)
+    norm = torch.empty_like(acc)
+    k_dev = torch.zeros(n_seq, dtype=torch.int32, device=dev)
+    idx = torch.empty(n_seq, L, dtype=torch.int32, device=dev)
+    out = torch.empty_like(batches[0][0])
+    kc = torch.empty(n_seq, L, Hkv, d, dtype=torch.bfloat16, device=dev)
+    vc = torch.empty_like(kc)
+    seq = torch.zeros(n_seq, dtype=torch.int32, device=dev)
+    st = torch.zeros(1, dtype=torch.int32, device=dev)
+    lay = z.zipvl_layer(L, Hq, Hkv, d, z.ZIPVL_BF16, 0, 0, 0, 0.0, 0)
+    ws_s = z.workspace(z.load().zipvl_workspace_bytes_batch(z.OP_SCORE, __import__("ctypes").byref(lay), 128, n_seq), dev)
+    ws_sel = z.workspace(z.zipvl_workspace_bytes(z.OP_SELECT, lay), dev)
+    ws_pf = z.workspace(z.zipvl_workspace_bytes(z.OP_SPARSE_PREFILL, lay), dev)
+    tau = layers[0].tau
+
+    def one(i):
+        q, k, v, probe = batches[i % 2]
+        z.zipvl_score_batch(q, k, probe, acc=acc, norm=norm, ws=ws_s, status=st)
+        z.zipvl_select_batch(acc, norm, tau, k_out=k_dev, idx=idx, ws=ws_sel, status=st)
+        z.zipvl_sparse_prefill_batch(q, k, v, idx, k_dev, L, kc, vc, L, out=out, len_out=seq, ws=ws_pf, status=st)
+
+    for i in range(4):
+        one(i)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(reps):
+        one(i)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / reps
+    ks = k_dev.cpu().numpy().astype(np.int64)
+    flops = float(np.sum(4.0 * d * Hq * ks * (ks + 1) / 2.0))
+    last = (reps - 1) % 2
+    chk = check_prefill_rows(batches[last][0][n_seq - 1], batches[last][1][n_seq - 1], batches[last][2][n_seq - 1],
+                             idx[n_seq - 1], k_dev[n_seq - 1:], out[n_seq - 1], seed=4)
+    return {"n_seq": n_seq, "ms_per_batch": ms, "ms_per_layer": ms / n_seq, "k": ks.tolist(),
+            "selected_tflops_per_s": flops / (ms * 1e-3) / 1e12,
+            "frac_of_bf16_burst_whole_prefill": flops / (ms * 1e-3) / 1e12 / peaks["tf_burst"],
+            "device_status_word": int(st.item()), "check": chk,
+            "note": "score + select + sparse prefill with compaction for 4 sequences per call (no decode step)"}
+
+
 def decode_benchmark(z, dev, steps, peaks, B=16, ctx_max=32768):
     """Batched decode on compacted caches (16 requests, contexts 4K-32K, 32 heads
     x 128, bf16) against the same kernel on the uncompacted caches."""
@@ -568,7 +622,7 @@ def run_ours(args, rank, world, local):
     t1e.record()
     torch.cuda.synchronize()
     est_ms = max(t0e.elapsed_time(t1e) / K, 1e-3)
-    repeats = max(1, int(math.ceil(MIN_REGION_MS / (est_ms * K))))
+    repeats = max(1, int(math.ceil(1.1 * MIN_REGION_MS / (est_ms * K))))
     n_ev = min(repeats * K, 400)
     events = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(n_ev)]
     events2 = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(K)]
@@ -707,6 +761,13 @@ def run_ours(args, rank, world, local):
         except Exception as e:  # report, never hide
             dec = {"error": repr(e)}
 
+    batched = None
+    if not args.no_batched:
+        try:
+            batched = batched_benchmark(z, dev, layers, peaks)
+        except Exception as e:  # report, never hide
+            batched = {"error": repr(e)}
+
     stack = None
     if args.stack_layers > 0:
         try:
@@ -765,7 +826,7 @@ def run_ours(args, rank, world, local):
         "graph_replay_ms_per_step": graph_ms,
         "prefill_ms": float(call_ms[0] + call_ms[1] + call_ms[2]),
         "prefill_tflops_selected": flops / (float(call_ms[0] + call_ms[1] + call_ms[2]) * 1e-3) / 1e12,
-        "roofline": roof, "other_kernels": others, "decode": dec, "stack": stack, "long_video": video, "library_context": context,
+        "roofline": roof, "other_kernels": others, "decode": dec, "batched": batched, "stack": stack, "long_video": video, "library_context": context,
         "cpu_baseline": cpu,
         "e2e": {"value": e2e_ms / world, "unit": "ms", "h2d_bytes_per_step": int(h2d),
                 "d2h_bytes_per_step": int(d2h),
@@ -788,6 +849,7 @@ def main():
                     help="largest context of the batched-decode leg (smaller = a light profiling case)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-long-video", action="store_true", help="skip the long-video (18K-token GQA) leg")
+    ap.add_argument("--no-batched", action="store_true", help="skip the 4-sequences-per-call leg")
     ap.add_argument("--library-context", action="store_true",
                     help="also time library attention (flash_attn) on gathered copies and dense, for context")
     ap.add_argument("--stack-layers", type=int, default=40,

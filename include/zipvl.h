@@ -231,6 +231,51 @@ zipvl_status zipvl_sparse_prefill_compact(const zipvl_layer *layer, const void *
                                           size_t ws_bytes, int32_t *status_word, void *stream);
 
 /*
+ * Several sequences per call.  (The paper treats one sequence; Algorithm 1 is run for every
+ * layer of every sequence, and sequences are independent, so a batch is the same arithmetic
+ * per sequence.)  A batch is n_seq sequences of ONE shape (the zipvl_layer), stacked:
+ * sequence z of Q starts q_stride_seq elements after sequence z-1 (0 = L x token stride,
+ * i.e. [n_seq, L, Hq, d] without gaps), K and V likewise with kv_stride_seq.  Everything
+ * per-sequence is stacked without gaps: probe_pos [n_seq, n_probe], acc / norm / idx
+ * [n_seq, L], k_out / k_dev / len_out / total / kept_mass [n_seq], out [n_seq, L or k_max,
+ * Hq, d], caches [n_seq, capacity, Hkv, d].  Results per sequence are those of the
+ * single-sequence calls, bit for bit.  Where the tensor-core kernels apply, a batch is one
+ * launch whose grid spans the sequences (short sequences alone cannot fill the GPU);
+ * other shapes run sequence by sequence inside the call.
+ */
+typedef struct {
+    int32_t n_seq;
+    int32_t reserved;
+    int64_t q_stride_seq;  /* elements between sequences of Q; 0 = L * token stride */
+    int64_t kv_stride_seq; /* elements between sequences of K and of V; 0 = L * token stride */
+} zipvl_batch;
+
+/* zipvl_workspace_bytes for the batched calls (only ZIPVL_OP_SCORE grows with n_seq). */
+size_t zipvl_workspace_bytes_batch(int32_t op, const zipvl_layer *layer, int32_t n_probe, int32_t n_seq);
+
+/* zipvl_score for a batch (Eq. A, Eq. 6, Eq. 8 per sequence). */
+zipvl_status zipvl_score_batch(const zipvl_layer *layer, const zipvl_batch *batch, const void *q,
+                               const void *k, const int32_t *probe_pos, int32_t n_probe, float *acc,
+                               float *norm, double *total, void *ws, size_t ws_bytes,
+                               int32_t *status_word, void *stream);
+
+/* zipvl_select for a batch of n_seq score rows of length L (Eq. 7, Eq. 9 per sequence; one
+ * tau, mode and fixed_k for all). */
+zipvl_status zipvl_select_batch(int32_t L, int32_t n_seq, const float *acc, const float *norm, float tau,
+                                uint32_t mode, int32_t fixed_k, int32_t *k_out, int32_t *idx,
+                                float *kept_mass, void *ws, size_t ws_bytes, int32_t *status_word,
+                                void *stream);
+
+/* zipvl_sparse_prefill for a batch (Algorithm 1's attention per sequence); with k_cache !=
+ * NULL also zipvl_compact_kv, as zipvl_sparse_prefill_compact does (then v_cache and len_out
+ * are required and capacity >= 1). */
+zipvl_status zipvl_sparse_prefill_batch(const zipvl_layer *layer, const zipvl_batch *batch, const void *q,
+                                        const void *k, const void *v, const int32_t *idx,
+                                        const int32_t *k_dev, int32_t k_max, void *out, int32_t out_mode,
+                                        void *k_cache, void *v_cache, int32_t capacity, int32_t *len_out,
+                                        void *ws, size_t ws_bytes, int32_t *status_word, void *stream);
+
+/*
  * zipvl_decode -- one decoding step over the kept cache, ragged batch.
  * Paper: Algorithm 2; Eq. 4 (append the new key / value), Eq. 5 (attention of
  * the single query over the whole cache).  Nothing is evicted while decoding.

@@ -24,7 +24,8 @@ DEV_BAD_INDEX, DEV_TIMEOUT, DEV_CAPACITY, DEV_BAD_VALUE = 1, 2, 4, 8
 EXPORTS = ["zipvl_status_string", "zipvl_last_error", "zipvl_version", "zipvl_launch_count",
            "zipvl_workspace_bytes",
            "zipvl_score", "zipvl_select", "zipvl_sparse_prefill", "zipvl_compact_kv",
-           "zipvl_sparse_prefill_compact",
+           "zipvl_sparse_prefill_compact", "zipvl_workspace_bytes_batch", "zipvl_score_batch",
+           "zipvl_select_batch", "zipvl_sparse_prefill_batch",
            "zipvl_decode", "zipvl_decode_paged", "zipvl_decode_noalloc", "zipvl_prefill_layer_host", "zipvl_layer_step_host",
            "zipvl_release_host_scratch", "zipvl_selftest_wait_timeout"]
 
@@ -45,6 +46,11 @@ class zipvl_layer(C.Structure):
 class zipvl_decode_desc(C.Structure):
     _fields_ = [("batch", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
                 ("head_dim", C.c_int32), ("dtype", C.c_int32), ("softmax_scale", C.c_float)]
+
+
+class zipvl_batch(C.Structure):
+    _fields_ = [("n_seq", C.c_int32), ("reserved", C.c_int32), ("q_stride_seq", C.c_int64),
+                ("kv_stride_seq", C.c_int64)]
 
 
 _lib = None
@@ -84,6 +90,16 @@ def load():
     lib.zipvl_decode.restype = C.c_int
     lib.zipvl_decode.argtypes = [C.POINTER(zipvl_decode_desc), vp, vp, vp, vp, vp, vp, vp, vp,
                                  i32, vp, vp, sz, vp, vp]
+    bp = C.POINTER(zipvl_batch)
+    lib.zipvl_workspace_bytes_batch.restype = sz
+    lib.zipvl_workspace_bytes_batch.argtypes = [i32, lp, i32, i32]
+    lib.zipvl_score_batch.restype = C.c_int
+    lib.zipvl_score_batch.argtypes = [lp, bp, vp, vp, vp, i32, vp, vp, vp, vp, sz, vp, vp]
+    lib.zipvl_select_batch.restype = C.c_int
+    lib.zipvl_select_batch.argtypes = [i32, i32, vp, vp, f32, u32, i32, vp, vp, vp, vp, sz, vp, vp]
+    lib.zipvl_sparse_prefill_batch.restype = C.c_int
+    lib.zipvl_sparse_prefill_batch.argtypes = [lp, bp, vp, vp, vp, vp, vp, i32, vp, i32, vp, vp, i32, vp,
+                                               vp, sz, vp, vp]
     lib.zipvl_decode_paged.restype = C.c_int
     lib.zipvl_decode_paged.argtypes = [C.POINTER(zipvl_decode_desc), vp, vp, vp, vp, vp, vp, i32, i32, i32,
                                        vp, vp, i32, vp, vp, sz, vp, vp]
@@ -236,6 +252,67 @@ def zipvl_sparse_prefill_compact(layer, q, k, v, idx, k_dev, k_max, k_cache, v_c
         C.byref(layer), _ptr(q), _ptr(k), _ptr(v), _ptr(idx), _ptr(k_dev), int(k_max), _ptr(out),
         out_mode, _ptr(k_cache), _ptr(v_cache), int(capacity), _ptr(len_out), _ptr(ws), ws.numel(),
         _ptr(status), _stream(stream)))
+    return out, len_out
+
+
+def _batch_desc(q, k):
+    """zipvl_layer + zipvl_batch for stacked Q [n_seq, L, Hq, d] and K [n_seq, L, Hkv, d]
+    (contiguous)."""
+    if q.dim() != 4 or not q.is_contiguous() or not k.is_contiguous():
+        raise ValueError("zipvl: batched calls take contiguous [n_seq, L, H, d] tensors")
+    n_seq, L, Hq, d = q.shape
+    lay = zipvl_layer(L, Hq, k.shape[2], d, _dtype_code(q), 0, 0, 0, 0.0, 0)
+    return lay, zipvl_batch(n_seq, 0, 0, 0)
+
+
+def zipvl_score_batch(q, k, probe_pos, acc=None, norm=None, ws=None, status=None, stream=None):
+    """zipvl_score for stacked sequences: q [n_seq,L,Hq,d], k [n_seq,L,Hkv,d], probe_pos int32
+    [n_seq,P]; returns (acc, norm) float32 [n_seq, L]."""
+    _dev(q, "q"), _dev(k, "k"), _dev(probe_pos, "probe_pos", torch.int32)
+    lay, b = _batch_desc(q, k)
+    n_seq, L, P = q.shape[0], q.shape[1], probe_pos.shape[1]
+    acc = torch.empty(n_seq, L, dtype=torch.float32, device=q.device) if acc is None else acc
+    norm = torch.empty(n_seq, L, dtype=torch.float32, device=q.device) if norm is None else norm
+    if ws is None:
+        ws = workspace(load().zipvl_workspace_bytes_batch(OP_SCORE, C.byref(lay), P, n_seq), q.device)
+    _check(load().zipvl_score_batch(C.byref(lay), C.byref(b), _ptr(q), _ptr(k), _ptr(probe_pos), P, _ptr(acc),
+                                    _ptr(norm), None, _ptr(ws), ws.numel(), _ptr(status), _stream(stream)))
+    return acc, norm
+
+
+def zipvl_select_batch(acc, norm, tau, mode=0, fixed_k=0, k_out=None, idx=None, ws=None, status=None,
+                       stream=None):
+    """zipvl_select for score rows [n_seq, L]; returns (k_out int32[n_seq], idx int32[n_seq, L])."""
+    _dev(acc, "acc", torch.float32), _dev(norm, "norm", torch.float32)
+    n_seq, L = acc.shape
+    k_out = torch.empty(n_seq, dtype=torch.int32, device=acc.device) if k_out is None else k_out
+    idx = torch.empty(n_seq, L, dtype=torch.int32, device=acc.device) if idx is None else idx
+    if ws is None:
+        lay = zipvl_layer(L, 1, 1, 64, ZIPVL_F32, 0, 0, 0, 0.0, 0)
+        ws = workspace(zipvl_workspace_bytes(OP_SELECT, lay), acc.device)
+    _check(load().zipvl_select_batch(L, n_seq, _ptr(acc), _ptr(norm), float(tau), mode, fixed_k, _ptr(k_out),
+                                     _ptr(idx), None, _ptr(ws), ws.numel(), _ptr(status), _stream(stream)))
+    return k_out, idx
+
+
+def zipvl_sparse_prefill_batch(q, k, v, idx, k_dev, k_max, k_cache=None, v_cache=None, capacity=0, out=None,
+                               out_mode=OUT_PADDED, len_out=None, ws=None, status=None, stream=None):
+    """zipvl_sparse_prefill (and, with caches, zipvl_compact_kv) for stacked sequences; returns
+    (out [n_seq, L or k_max, Hq, d], len_out or None)."""
+    _dev(q, "q"), _dev(k, "k"), _dev(v, "v"), _dev(idx, "idx", torch.int32), _dev(k_dev, "k_dev", torch.int32)
+    lay, b = _batch_desc(q, k)
+    n_seq, L = q.shape[0], q.shape[1]
+    if out is None:
+        rows = L if out_mode == OUT_PADDED else k_max
+        out = torch.empty((n_seq, rows, lay.n_q_heads, lay.head_dim), dtype=q.dtype, device=q.device)
+    if ws is None:
+        ws = workspace(zipvl_workspace_bytes(OP_SPARSE_PREFILL, lay), q.device)
+    if k_cache is not None and len_out is None:
+        len_out = torch.empty(n_seq, dtype=torch.int32, device=q.device)
+    _check(load().zipvl_sparse_prefill_batch(C.byref(lay), C.byref(b), _ptr(q), _ptr(k), _ptr(v), _ptr(idx),
+                                             _ptr(k_dev), int(k_max), _ptr(out), out_mode, _ptr(k_cache),
+                                             _ptr(v_cache), int(capacity), _ptr(len_out), _ptr(ws), ws.numel(),
+                                             _ptr(status), _stream(stream)))
     return out, len_out
 
 

@@ -55,6 +55,7 @@ static zipvl_status check_layer(const char *who, const zipvl_layer *l, LayerArgs
     const float scale = l->softmax_scale > 0.f ? l->softmax_scale : 1.0f / sqrtf((float)l->head_dim);
     a->scale_log2 = scale * kLog2e;
     a->half = (l->dtype == ZIPVL_F16);
+    a->n_seq = 1; a->q_seq = 0; a->kv_seq = 0;
     return ZIPVL_OK;
 }
 
@@ -250,6 +251,131 @@ zipvl_status zipvl_decode(const zipvl_decode_desc *d, const void *q, const void 
     const float scale = d->softmax_scale > 0.f ? d->softmax_scale : 1.0f / sqrtf((float)d->head_dim);
     return launch_decode(*d, scale * kLog2e, q, k_new, v_new, k_cache, v_cache, cache_off, capacity,
                          seq_lens, max_len, out, ws, status_word, (cudaStream_t)stream);
+}
+
+// ---- several sequences of one shape per call -------------------------------------------
+static zipvl_status check_batch(const char *who, const zipvl_batch *b, const LayerArgs &a, long long *q_seq,
+                                long long *kv_seq) {
+    if (!b) return fail(ZIPVL_ERR_INVALID_ARG, "%s: batch is NULL", who);
+    if (b->n_seq < 1 || b->n_seq > 4096) return fail(ZIPVL_ERR_INVALID_ARG, "%s: n_seq = %d", who, b->n_seq);
+    *q_seq = b->q_stride_seq ? b->q_stride_seq : (long long)a.L * a.q_stride;
+    *kv_seq = b->kv_stride_seq ? b->kv_stride_seq : (long long)a.L * a.kv_stride;
+    if (*q_seq < (long long)a.L * a.q_stride || *kv_seq < (long long)a.L * a.kv_stride || *q_seq % 8 || *kv_seq % 8)
+        return fail(ZIPVL_ERR_INVALID_ARG, "%s: sequence strides %lld / %lld", who, *q_seq, *kv_seq);
+    return ZIPVL_OK;
+}
+
+size_t zipvl_workspace_bytes_batch(int32_t op, const zipvl_layer *layer, int32_t n_probe, int32_t n_seq) {
+    LayerArgs a{};
+    if (n_seq < 1 || check_layer("workspace_bytes_batch", layer, &a) != ZIPVL_OK) return 0;
+    if (op == ZIPVL_OP_SCORE) {
+        if (n_probe < 1) return 0;
+        return align256(score_simt_ws_bytes(a.L, a.Hq, n_probe)) +
+               align256(score_tc_ws_bytes(a.L, a.Hq, a.Hkv, n_probe, n_seq));
+    }
+    return zipvl_workspace_bytes(op, layer, n_probe, 1);
+}
+
+zipvl_status zipvl_score_batch(const zipvl_layer *layer, const zipvl_batch *batch, const void *q,
+                               const void *k, const int32_t *probe_pos, int32_t n_probe, float *acc,
+                               float *norm, double *total, void *ws, size_t ws_bytes,
+                               int32_t *status_word, void *stream) {
+    LayerArgs a{};
+    zipvl_status s = check_layer("zipvl_score_batch", layer, &a);
+    if (s != ZIPVL_OK) return s;
+    long long q_seq = 0, kv_seq = 0;
+    s = check_batch("zipvl_score_batch", batch, a, &q_seq, &kv_seq);
+    if (s != ZIPVL_OK) return s;
+    if (!q || !k || !probe_pos || !acc || !norm || !ws)
+        return fail(ZIPVL_ERR_INVALID_ARG, "zipvl_score_batch: NULL pointer");
+    if (n_probe < 1) return fail(ZIPVL_ERR_INVALID_ARG, "zipvl_score_batch: n_probe = %d", n_probe);
+    if (!aligned16(q) || !aligned16(k) || !aligned16(ws))
+        return fail(ZIPVL_ERR_INVALID_ARG, "zipvl_score_batch: q, k, ws must be 16-byte aligned");
+    const size_t need = zipvl_workspace_bytes_batch(ZIPVL_OP_SCORE, layer, n_probe, batch->n_seq);
+    if (ws_bytes < need) return fail(ZIPVL_ERR_WORKSPACE, "zipvl_score_batch: workspace %zu < %zu", ws_bytes, need);
+    // one launch pair for the whole batch when the tensor-core kernels apply and K is stacked
+    // without gaps (one tensor map of n_seq * L rows); otherwise sequence by sequence
+    if (score_tc_supported(a, layer->dtype, n_probe) && kv_seq == (long long)a.L * a.kv_stride) {
+        a.n_seq = batch->n_seq; a.q_seq = q_seq; a.kv_seq = kv_seq;
+        return launch_score_tc(a, q, k, probe_pos, n_probe, acc, norm, total, ws, status_word,
+                               (cudaStream_t)stream);
+    }
+    const size_t eb = elem_bytes(layer->dtype);
+    for (int z = 0; z < batch->n_seq; ++z) {
+        s = zipvl_score(layer, (const char *)q + (size_t)z * q_seq * eb, (const char *)k + (size_t)z * kv_seq * eb,
+                        probe_pos + (size_t)z * n_probe, n_probe, acc + (size_t)z * a.L, norm + (size_t)z * a.L,
+                        total ? total + z : nullptr, ws, ws_bytes, status_word, stream);
+        if (s != ZIPVL_OK) return s;
+    }
+    return ZIPVL_OK;
+}
+
+zipvl_status zipvl_select_batch(int32_t L, int32_t n_seq, const float *acc, const float *norm, float tau,
+                                uint32_t mode, int32_t fixed_k, int32_t *k_out, int32_t *idx,
+                                float *kept_mass, void *ws, size_t ws_bytes, int32_t *status_word,
+                                void *stream) {
+    if (n_seq < 1 || n_seq > 4096) return fail(ZIPVL_ERR_INVALID_ARG, "zipvl_select_batch: n_seq = %d", n_seq);
+    if (L < 1 || L > kMaxSelectL) return fail(ZIPVL_ERR_INVALID_ARG, "zipvl_select_batch: L = %d", L);
+    if (!acc || !norm || !k_out || !idx) return fail(ZIPVL_ERR_INVALID_ARG, "zipvl_select_batch: NULL pointer");
+    if (!(tau > 0.f && tau <= 1.f)) return fail(ZIPVL_ERR_INVALID_ARG, "zipvl_select_batch: tau = %g not in (0,1]", (double)tau);
+    if (fixed_k < 0) return fail(ZIPVL_ERR_INVALID_ARG, "zipvl_select_batch: fixed_k = %d", fixed_k);
+    if (mode & 0xFFu & ~(ZIPVL_BUDGET_BY_NORM | ZIPVL_TOPK_BY_ACC))
+        return fail(ZIPVL_ERR_INVALID_ARG, "zipvl_select_batch: mode = %u", mode);
+    if (!ws || ws_bytes < select_ws_bytes())
+        return fail(ZIPVL_ERR_WORKSPACE, "zipvl_select_batch: workspace %zu < %zu", ws_bytes, select_ws_bytes());
+    if (!aligned16(ws)) return fail(ZIPVL_ERR_INVALID_ARG, "zipvl_select_batch: ws must be 16-byte aligned");
+    return launch_select(L, acc, norm, tau, mode, fixed_k, k_out, idx, kept_mass, ws, status_word,
+                         (cudaStream_t)stream, n_seq);
+}
+
+zipvl_status zipvl_sparse_prefill_batch(const zipvl_layer *layer, const zipvl_batch *batch, const void *q,
+                                        const void *k, const void *v, const int32_t *idx,
+                                        const int32_t *k_dev, int32_t k_max, void *out, int32_t out_mode,
+                                        void *k_cache, void *v_cache, int32_t capacity, int32_t *len_out,
+                                        void *ws, size_t ws_bytes, int32_t *status_word, void *stream) {
+    const char *who = "zipvl_sparse_prefill_batch";
+    LayerArgs a{};
+    zipvl_status s = check_layer(who, layer, &a);
+    if (s != ZIPVL_OK) return s;
+    long long q_seq = 0, kv_seq = 0;
+    s = check_batch(who, batch, a, &q_seq, &kv_seq);
+    if (s != ZIPVL_OK) return s;
+    if (!q || !k || !v || !idx || !k_dev || !out) return fail(ZIPVL_ERR_INVALID_ARG, "%s: NULL pointer", who);
+    const bool caches = (k_cache != nullptr);
+    if (caches && (!v_cache || !len_out || capacity < 1))
+        return fail(ZIPVL_ERR_INVALID_ARG, "%s: k_cache needs v_cache, len_out and capacity >= 1", who);
+    if (k_max < 1 || k_max > a.L) return fail(ZIPVL_ERR_INVALID_ARG, "%s: k_max = %d not in [1, L]", who, k_max);
+    if (out_mode != ZIPVL_OUT_PADDED && out_mode != ZIPVL_OUT_COMPACT)
+        return fail(ZIPVL_ERR_INVALID_ARG, "%s: out_mode = %d", who, out_mode);
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) ||
+        (caches && (!aligned16(k_cache) || !aligned16(v_cache))))
+        return fail(ZIPVL_ERR_INVALID_ARG, "%s: tensors must be 16-byte aligned", who);
+    if (prefill_tc_supported(a, layer->dtype) && a.kv_stride % 8 == 0) {
+        if (!ws || ws_bytes < zipvl_workspace_bytes(ZIPVL_OP_SPARSE_PREFILL, layer, 0, 1))
+            return fail(ZIPVL_ERR_WORKSPACE, "%s: workspace %zu < %zu", who, ws_bytes,
+                        zipvl_workspace_bytes(ZIPVL_OP_SPARSE_PREFILL, layer, 0, 1));
+        a.n_seq = batch->n_seq; a.q_seq = q_seq; a.kv_seq = kv_seq;
+        return launch_prefill_tc(a, q, k, v, idx, k_dev, k_max, out, out_mode, k_cache, v_cache, capacity,
+                                 len_out, ws, status_word, (cudaStream_t)stream);
+    }
+    // other shapes and types: sequence by sequence through the single-sequence calls
+    const size_t eb = elem_bytes(layer->dtype);
+    const size_t out_seq = (size_t)(out_mode == ZIPVL_OUT_PADDED ? a.L : k_max) * a.Hq * a.D * eb;
+    const size_t cache_seq = (size_t)capacity * a.Hkv * a.D * eb;
+    for (int z = 0; z < batch->n_seq; ++z) {
+        const char *qz = (const char *)q + (size_t)z * q_seq * eb;
+        const char *kz = (const char *)k + (size_t)z * kv_seq * eb, *vz = (const char *)v + (size_t)z * kv_seq * eb;
+        if (caches)
+            s = zipvl_sparse_prefill_compact(layer, qz, kz, vz, idx + (size_t)z * a.L, k_dev + z, k_max,
+                                             (char *)out + z * out_seq, out_mode, (char *)k_cache + z * cache_seq,
+                                             (char *)v_cache + z * cache_seq, capacity, len_out + z, ws, ws_bytes,
+                                             status_word, stream);
+        else
+            s = zipvl_sparse_prefill(layer, qz, kz, vz, idx + (size_t)z * a.L, k_dev + z, k_max,
+                                     (char *)out + z * out_seq, out_mode, ws, ws_bytes, status_word, stream);
+        if (s != ZIPVL_OK) return s;
+    }
+    return ZIPVL_OK;
 }
 
 #define ZIPVL_CUDA(call)                                                                   \

@@ -117,6 +117,10 @@ struct LayerArgs {
     long long q_stride, kv_stride;  // elements per token
     float scale_log2;               // softmax scale * log2(e)
     int half;                       // 16-bit storage is IEEE half (1) or bfloat16 (0)
+    // a batch of n_seq sequences of this shape (1 for the single-sequence calls): elements
+    // between the sequences of Q and of K / V; per-sequence outputs are stacked likewise
+    int n_seq;
+    long long q_seq, kv_seq;
 };
 
 zipvl_status launch_score_simt(const LayerArgs &a, int dtype, const void *q, const void *k,
@@ -126,7 +130,7 @@ size_t score_simt_ws_bytes(int L, int Hq, int P);
 
 zipvl_status launch_select(int L, const float *acc, const float *norm, float tau, uint32_t mode,
                            int fixed_k, int32_t *k_out, int32_t *idx, float *kept_mass, void *ws,
-                           int32_t *status_word, cudaStream_t st);
+                           int32_t *status_word, cudaStream_t st, int n_seq = 1);
 size_t select_ws_bytes();
 
 zipvl_status launch_prefill_simt(const LayerArgs &a, int dtype, const void *q, const void *k,

@@ -147,9 +147,24 @@ prefill_tc_kernel(LayerArgs a, const __nv_bfloat16 *__restrict__ q,
     }
     if (warp == 12) tmem_alloc(smem_u32(&bar->tmem_base), kTmemCols);
     grid_dependency_wait(q, k, v, idx, k_dev);   // k_dev and idx are the previous kernel's output
+    // grid.x = query head + Hq * sequence: every sequence of a batch has its own tensors, index
+    // list, k, output and cache, stacked; its heaviest pairs still start first
+    const int h = blockIdx.x % a.Hq, g = h / a.G;
+    {
+        const int z = blockIdx.x / a.Hq;
+        q += z * a.q_seq; k += z * a.kv_seq; v += z * a.kv_seq;
+        idx += (long long)z * a.L;
+        k_dev += z;
+        out += (long long)z * (out_mode == ZIPVL_OUT_PADDED ? a.L : k_max) * a.Hq * kD;
+        if (kc != nullptr) {
+            kc += (long long)z * capacity * a.Hkv * kD;
+            vc += (long long)z * capacity * a.Hkv * kD;
+            len_out += z;
+        }
+    }
     int n_valid = *k_dev;
     if (n_valid > k_max || n_valid < 0) {
-        if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0)
+        if (h == 0 && blockIdx.y == 0 && threadIdx.x == 0)
             report(status_word, ZIPVL_DEV_CAPACITY);
         n_valid = n_valid < 0 ? 0 : k_max;
     }
@@ -167,8 +182,7 @@ prefill_tc_kernel(LayerArgs a, const __nv_bfloat16 *__restrict__ q,
     const int pt = n_pairs - 1 - (int)blockIdx.y;
     const int ta = pt > 0 ? 2 * pt - odd : 0;       // tile A of this CTA (tile B = ta + 1)
     const int q0 = ta * kBM;
-    const bool no_work = (pt < 0 || q0 >= n_valid || (int)blockIdx.x >= a.Hq);   // or a bad grid
-    const int h = blockIdx.x, g = h / a.G;
+    const bool no_work = (pt < 0 || q0 >= n_valid || (int)blockIdx.x >= a.Hq * a.n_seq);   // or a bad grid
     const bool has_b = !(odd && pt == 0) && (q0 + kBM) < n_valid;   // tile B exists and has a valid row
     const int n_a = ta + 1;                         // key tiles of A (diagonal = ta)
     const int n_kv = has_b ? n_a + 1 : n_a;         // key tiles of B (diagonal = ta + 1)
@@ -193,7 +207,7 @@ prefill_tc_kernel(LayerArgs a, const __nv_bfloat16 *__restrict__ q,
     const uint32_t tmem = bar->tmem_base;
     if (no_work) {                                  // a CTA past the kept set: give the columns back
         if (warp == 12) tmem_dealloc(tmem, kTmemCols);
-        if (n_valid == 0 && blockIdx.y == 0 && (int)blockIdx.x < a.Hq) {
+        if (n_valid == 0 && blockIdx.y == 0 && (int)blockIdx.x < a.Hq * a.n_seq) {
             // nothing kept: the results are those of the two separate calls -- an all-zero
             // PADDED output (every row is a dropped token's) and a cache of length 0
             if (out_mode == ZIPVL_OUT_PADDED) {
@@ -201,7 +215,7 @@ prefill_tc_kernel(LayerArgs a, const __nv_bfloat16 *__restrict__ q,
                 for (int e = threadIdx.x; e < a.L * 16; e += kThreadsTc)
                     reinterpret_cast<uint4 *>(out + ((long long)(e >> 4) * a.Hq + h) * kD)[e & 15] = z;
             }
-            if (kc != nullptr && blockIdx.x == 0 && threadIdx.x == 0) *len_out = 0;
+            if (kc != nullptr && h == 0 && threadIdx.x == 0) *len_out = 0;
         }
         return;
     }
@@ -311,7 +325,7 @@ prefill_tc_kernel(LayerArgs a, const __nv_bfloat16 *__restrict__ q,
                         }
                     }
                 }
-                if (blockIdx.x == 0 && blockIdx.y == 0 && warp == 13 && lane == 0) {
+                if (h == 0 && blockIdx.y == 0 && warp == 13 && lane == 0) {
                     *len_out = lim;
                     if (n_valid > capacity) report(status_word, ZIPVL_DEV_CAPACITY);
                 }
@@ -618,14 +632,14 @@ zipvl_status launch_prefill_tc(const LayerArgs &a, const void *q, const void *k,
     const char *env = getenv("ZIPVL_PREFILL_KERNEL");
     const int forced = !env ? 0 : (!strcmp(env, "pair") ? 1 : (!strcmp(env, "single") ? 2 : 0));
     const bool single = forced ? (forced == 2) : ((long long)k_max * a.Hq <= kSingleTileMaxRows);
-    if (single)
+    if (single && a.n_seq == 1)
         return launch_prefill_tc1(a, q, k, v, idx, k_dev, k_max, out, out_mode, k_cache, v_cache,
                                   capacity, len_out, status_word, st);
     auto kernel = a.half ? prefill_tc_kernel<true> : prefill_tc_kernel<false>;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
     if (e != cudaSuccess)
         return fail(ZIPVL_ERR_CUDA, "sparse_prefill: smem opt-in: %s", cudaGetErrorString(e));
-    dim3 grid(a.Hq, (k_max + kPair - 1) / kPair);
+    dim3 grid(a.Hq * a.n_seq, (k_max + kPair - 1) / kPair);
     e = launch_dependent(kernel, grid, dim3(kThreadsTc), kSmemBytes, st, a, (const __nv_bfloat16 *)q,
                          (const __nv_bfloat16 *)k, (const __nv_bfloat16 *)v, idx, k_dev, k_max,
                          (__nv_bfloat16 *)out, out_mode, (__nv_bfloat16 *)k_cache,

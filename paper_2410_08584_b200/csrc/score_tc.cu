@@ -78,7 +78,16 @@ score_tc_kernel(const __grid_constant__ CUtensorMap kmap, LayerArgs a,
     ScBarriers *bar = reinterpret_cast<ScBarriers *>(sPos + kMaxProbe);
     volatile int *abort_flag = &bar->abort_flag;
 
-    const int chunk = blockIdx.x, h = blockIdx.y, g = h / a.G;
+    // blockIdx.z = sequence of a batch: its own probe rows, statistics, partial sums, counters
+    // and scores, stacked; K of all sequences is one tensor map of n_seq * L rows
+    const int chunk = blockIdx.x, h = blockIdx.y, g = h / a.G, z = blockIdx.z;
+    q += z * a.q_seq;
+    probe_pos += (long long)z * P;
+    stats += (long long)z * a.Hq * n_chunks * kMaxProbe;
+    partial += (long long)z * a.Hq * a.L;
+    counters += z * n_chunks;
+    acc += (long long)z * a.L;
+    norm += (long long)z * a.L;
     const int n_tiles_all = (a.L + kTile - 1) / kTile;
     const int t0 = chunk * tiles_per_chunk;
     const int t1 = min(n_tiles_all, t0 + tiles_per_chunk);
@@ -136,7 +145,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap kmap, LayerArgs a,
                 const uint32_t fb = smem_u32(&bar->k_full[s]);
                 mbar_expect_tx(fb, kTileBytes);
                 const uint32_t dst = sK + s * kTileBytes;
-                const int y = (t0 + n) * kTile;
+                const int y = z * a.L + (t0 + n) * kTile;
                 tma_load_2d(dst, &kmap, g * kD, y, fb);
                 tma_load_2d(dst + kHalfBytes, &kmap, g * kD + 64, y, fb);
             }
@@ -390,32 +399,34 @@ bool score_tc_supported(const LayerArgs &a, int dtype, int n_probe) {
            encode_tiled_fn() != nullptr;
 }
 
-size_t score_tc_ws_bytes(int L, int Hq, int, int) {
+size_t score_tc_ws_bytes(int L, int Hq, int, int, int n_seq) {
     const int n_tiles = (L + kTile - 1) / kTile;
-    const int tpc = tiles_per_chunk_for(L, Hq);
+    const int tpc = tiles_per_chunk_for(L, Hq * n_seq);
     const size_t n_chunks = (n_tiles + tpc - 1) / tpc;
     size_t stats = (size_t)Hq * n_chunks * kMaxProbe * sizeof(float2);
     stats = (stats + 255) & ~(size_t)255;
-    const size_t partial = ((size_t)Hq * L * sizeof(float) + 255) & ~(size_t)255;
-    return stats + partial + n_chunks * sizeof(int);
+    stats = ((stats * n_seq) + 255) & ~(size_t)255;
+    const size_t partial = ((size_t)n_seq * Hq * L * sizeof(float) + 255) & ~(size_t)255;
+    return stats + partial + n_seq * n_chunks * sizeof(int);
 }
 
 zipvl_status launch_score_tc(const LayerArgs &a, const void *q, const void *k,
                              const int32_t *probe_pos, int P, float *acc, float *norm,
                              double *total, void *ws, int32_t *status_word, cudaStream_t st) {
     const int n_tiles = (a.L + kTile - 1) / kTile;
-    const int tpc = tiles_per_chunk_for(a.L, a.Hq);
+    const int tpc = tiles_per_chunk_for(a.L, a.Hq * a.n_seq);
     const int n_chunks = (n_tiles + tpc - 1) / tpc;
-    size_t stats_bytes = (size_t)a.Hq * n_chunks * kMaxProbe * sizeof(float2);
+    size_t stats_bytes = (size_t)a.n_seq * a.Hq * n_chunks * kMaxProbe * sizeof(float2);
     stats_bytes = (stats_bytes + 255) & ~(size_t)255;
     float2 *stats = reinterpret_cast<float2 *>(ws);
     float *partial = reinterpret_cast<float *>(reinterpret_cast<char *>(ws) + stats_bytes);
-    const size_t partial_bytes = ((size_t)a.Hq * a.L * sizeof(float) + 255) & ~(size_t)255;
+    const size_t partial_bytes = ((size_t)a.n_seq * a.Hq * a.L * sizeof(float) + 255) & ~(size_t)255;
     int *counters = reinterpret_cast<int *>(reinterpret_cast<char *>(ws) + stats_bytes + partial_bytes);
 
     // tensor map over K viewed as [L rows, Hkv*d columns], box = 64 columns x 128 rows
     CUtensorMap kmap;
-    const cuuint64_t dims[2] = {(cuuint64_t)a.Hkv * a.D, (cuuint64_t)a.L};
+    // (a batch is stacked without gaps -- the caller checks -- so its K is one 2-D tensor)
+    const cuuint64_t dims[2] = {(cuuint64_t)a.Hkv * a.D, (cuuint64_t)a.L * a.n_seq};
     const cuuint64_t strides[1] = {(cuuint64_t)a.kv_stride * 2};
     const cuuint32_t box[2] = {64, (cuuint32_t)kTile};
     const cuuint32_t estr[2] = {1, 1};
@@ -432,7 +443,7 @@ zipvl_status launch_score_tc(const LayerArgs &a, const void *q, const void *k,
     if (e != cudaSuccess) return fail(ZIPVL_ERR_CUDA, "score: smem opt-in: %s", cudaGetErrorString(e));
 
     const __nv_bfloat16 *qb = (const __nv_bfloat16 *)q;
-    dim3 grid(n_chunks, a.Hq);
+    dim3 grid(n_chunks, a.Hq, a.n_seq);
     // both launches are programmatic dependents: <1> may begin its set-up, loads and first
     // MMA while <0> drains, and <0> itself may be staged behind the caller's previous kernel
     e = launch_dependent(score_tc_kernel<0>, grid, dim3(kThreadsSc), kScSmem, st, kmap, a, qb, probe_pos, P,
@@ -441,8 +452,9 @@ zipvl_status launch_score_tc(const LayerArgs &a, const void *q, const void *k,
         e = launch_dependent(score_tc_kernel<1>, grid, dim3(kThreadsSc), kScSmem, st, kmap, a, qb, probe_pos,
                              P, tpc, n_chunks, stats, partial, counters, acc, norm, status_word);
     if (e != cudaSuccess) return fail(ZIPVL_ERR_CUDA, "score: launch: %s", cudaGetErrorString(e));
-    if (total) sum_to_double_kernel<<<1, 1024, 0, st>>>(a.L, acc, total);
-    count_launches(total ? 3 : 2);
+    if (total)
+        for (int z = 0; z < a.n_seq; ++z) sum_to_double_kernel<<<1, 1024, 0, st>>>(a.L, acc + (size_t)z * a.L, total + z);
+    count_launches(total ? 2 + a.n_seq : 2);
     return check_launch("zipvl_score");
 }
 

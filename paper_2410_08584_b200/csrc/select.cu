@@ -799,6 +799,12 @@ select_solo_kernel(int L, const float *__restrict__ acc, const float *__restrict
     clear(&sm, sizeof(SoloSmem));      // while the previous kernel may still be running
     grid_launch_dependents();
     grid_dependency_wait(acc, norm);   // the scores are the previous kernel's output
+    // one CTA per sequence of a batch: score rows, index lists and results are stacked
+    acc += (size_t)blockIdx.x * L;
+    norm += (size_t)blockIdx.x * L;
+    idx += (size_t)blockIdx.x * L;
+    k_out += blockIdx.x;
+    if (kept_mass) kept_mass += blockIdx.x;
     const bool bud_is_norm = (mode & ZIPVL_BUDGET_BY_NORM) != 0, rank_is_acc = (mode & ZIPVL_TOPK_BY_ACC) != 0;
     // ---- the row into registers: positions j0 .. j0+15 (a vector that is not 16-byte aligned
     // is read element by element) ----
@@ -1021,13 +1027,23 @@ size_t select_ws_bytes() { return (sizeof(GlobalHist) + 255) & ~(size_t)255; }
 
 zipvl_status launch_select(int L, const float *acc, const float *norm, float tau, uint32_t mode,
                            int fixed_k, int32_t *k_out, int32_t *idx, float *kept_mass, void *ws,
-                           int32_t *status_word, cudaStream_t st) {
+                           int32_t *status_word, cudaStream_t st, int n_seq) {
+    if (L > kSoloMax && n_seq > 1) {
+        // long rows: the multi-CTA kernel takes one sequence at a time (its workspace too)
+        for (int z = 0; z < n_seq; ++z) {
+            const zipvl_status sz = launch_select(L, acc + (size_t)z * L, norm + (size_t)z * L, tau, mode, fixed_k,
+                                                  k_out + z, idx + (size_t)z * L, kept_mass ? kept_mass + z : nullptr,
+                                                  ws, status_word, st, 1);
+            if (sz != ZIPVL_OK) return sz;
+        }
+        return ZIPVL_OK;
+    }
     if (L <= kSoloMax) {
         auto solo = (mode >> 8) ? select_solo_kernel<true> : select_solo_kernel<false>;
         cudaError_t es = cudaFuncSetAttribute(solo, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                               (int)sizeof(SoloSmem));
         if (es == cudaSuccess)
-            es = launch_dependent(solo, dim3(1), dim3(kSoloThreads), sizeof(SoloSmem), st, L, acc, norm, tau,
+            es = launch_dependent(solo, dim3(n_seq), dim3(kSoloThreads), sizeof(SoloSmem), st, L, acc, norm, tau,
                                   mode, fixed_k, k_out, idx, kept_mass, status_word);
         if (es != cudaSuccess) return fail(ZIPVL_ERR_CUDA, "select: launch: %s", cudaGetErrorString(es));
         count_launches(1);

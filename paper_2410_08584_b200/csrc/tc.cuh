@@ -5,7 +5,7 @@
 namespace zipvl {
 
 bool score_tc_supported(const LayerArgs &a, int dtype, int n_probe);
-size_t score_tc_ws_bytes(int L, int Hq, int Hkv, int n_probe);
+size_t score_tc_ws_bytes(int L, int Hq, int Hkv, int n_probe, int n_seq = 1);
 zipvl_status launch_score_tc(const LayerArgs &a, const void *q, const void *k,
                              const int32_t *probe_pos, int P, float *acc, float *norm,
                              double *total, void *ws, int32_t *status_word, cudaStream_t st);

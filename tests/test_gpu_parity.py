@@ -227,6 +227,73 @@ def test_single_tile_attention_kernel_gives_the_bits_of_the_default_one(zipvl, n
     assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1]) and torch.equal(a[2], b[2])
 
 
+@pytest.mark.parametrize("kind", ["bf16_tensor_core", "fp16_gqa", "fp32_cuda_core"])
+def test_batched_calls_equal_the_single_sequence_calls(zipvl, kind):
+    """Several sequences of one shape through zipvl_score_batch / zipvl_select_batch /
+    zipvl_sparse_prefill_batch: per sequence the bits of the single-sequence calls (which the
+    tests above hold against the oracle), and sequence 0 once more against the oracle itself."""
+    if kind == "bf16_tensor_core":
+        layers = [W.heavy_key_layer(L_visual=700, L_text=64, H=4, seed=51 + i, probe_seed=500 + i,
+                                    heavy_frac=0.05 + 0.1 * i) for i in range(3)]
+    elif kind == "fp16_gqa":
+        layers = [W.video_layer(n_frames=5, Hq=14, Hkv=2, seed=61 + i, dtype=torch.float16) for i in range(2)]
+    else:
+        layers = [W.tiny_layer(L=333, H=2, d=64, n_probe=40, seed=71 + i) for i in range(2)]
+    n_seq, L = len(layers), layers[0].L
+    q = torch.stack([l.q for l in layers]).to(DEV)
+    k = torch.stack([l.k for l in layers]).to(DEV)
+    v = torch.stack([l.v for l in layers]).to(DEV)
+    probe = torch.stack([l.probe_pos for l in layers]).to(DEV)
+    tau = layers[0].tau
+    st = status_word()
+    acc, norm = zipvl.zipvl_score_batch(q, k, probe, status=st)
+    k_dev, idx = zipvl.zipvl_select_batch(acc, norm, tau, status=st)
+    Hkv, d = k.shape[2], k.shape[3]
+    cap = L + 3
+    kc = torch.zeros(n_seq, cap, Hkv, d, dtype=k.dtype, device=DEV)
+    vc = torch.zeros_like(kc)
+    out, n = zipvl.zipvl_sparse_prefill_batch(q, k, v, idx, k_dev, L, kc, vc, cap, status=st)
+    out_c, _ = zipvl.zipvl_sparse_prefill_batch(q, k, v, idx, k_dev, L, out_mode=zipvl.OUT_COMPACT, status=st)
+    torch.cuda.synchronize()
+    assert st.item() == 0
+    ks = k_dev.tolist()
+    assert len(set(ks)) > 1 or n_seq == 1, "the sequences should keep different numbers of tokens"
+    for z in range(n_seq):
+        desc = zipvl.layer_desc(q[z], k[z])
+        a1, n1 = zipvl.zipvl_score(desc, q[z], k[z], probe[z])
+        kd1, idx1 = zipvl.zipvl_select(a1, n1, tau)
+        kc1, vc1 = torch.zeros(cap, Hkv, d, dtype=k.dtype, device=DEV), torch.zeros(cap, Hkv, d, dtype=k.dtype, device=DEV)
+        o1, len1 = zipvl.zipvl_sparse_prefill_compact(desc, q[z], k[z], v[z], idx1, kd1, L, kc1, vc1, cap)
+        oc1 = zipvl.zipvl_sparse_prefill(desc, q[z], k[z], v[z], idx1, kd1, L, out_mode=zipvl.OUT_COMPACT)
+        torch.cuda.synchronize()
+        assert torch.equal(acc[z], a1) and torch.equal(norm[z], n1)
+        assert kd1.item() == ks[z] and torch.equal(idx[z], idx1)
+        assert torch.equal(out[z], o1) and n[z].item() == len1.item() == ks[z]
+        assert torch.equal(kc[z], kc1) and torch.equal(vc[z], vc1)
+        assert torch.equal(out_c[z][:ks[z]], oc1[:ks[z]])
+    # sequence 0 against the oracle
+    l0 = layers[0]
+    qf, kf, vf = to_np(l0.q), to_np(l0.k), to_np(l0.v)
+    acc_ref, S = oracle.probe_scores(qf, kf, l0.probe_pos.numpy())
+    norm_ref, _ = oracle.normalise(acc_ref, l0.probe_pos.numpy(), l0.n_q_heads)
+    check_scores(acc[0].cpu().numpy(), norm[0].cpu().numpy(), acc_ref, norm_ref, S)
+    T = idx[0][:ks[0]].cpu().numpy()
+    ref = oracle.sparse_prefill(qf, kf, vf, T)
+    check_attention(to_np(out[0])[T], ref, l0.q.dtype)
+
+
+def test_batched_select_of_long_rows(zipvl):
+    """Rows longer than one CTA holds go through the multi-CTA kernel sequence by sequence."""
+    g = torch.Generator().manual_seed(9)
+    acc = (torch.rand(3, 5000, generator=g) ** 3).to(DEV)
+    norm = (acc.cpu() * torch.rand(3, 5000, generator=g)).to(DEV)
+    k_dev, idx = zipvl.zipvl_select_batch(acc, norm, 0.9)
+    torch.cuda.synchronize()
+    for z in range(3):
+        check_select(int(k_dev[z].item()), idx[z].cpu().numpy(), acc[z].cpu().numpy().astype(np.float64),
+                     norm[z].cpu().numpy().astype(np.float64), 0.9)
+
+
 def test_fused_prefill_compaction_reports_a_small_cache(zipvl):
     layer = CASES["llava7b_small_bf16"]()
     q, k, v, probe = put(layer)
