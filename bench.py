@@ -285,12 +285,12 @@ def check_prefill_rows(layer_q, layer_k, layer_v, idx, k_dev, out, n_rows=32, se
             "max_abs": float(d.max()), "mean_abs": float(d.mean())}
 
 
-def long_video_benchmark(z, dev, peaks, reps=10):
+def long_video_benchmark(z, dev, peaks, reps=10, taus=(0.95, 0.99), sustained=250):
     """Long-video GQA layer (L 18432 = 128 frames x 144 tokens, 28 query / 4 KV heads) at
     tau 0.95 and 0.99: per-call times of score, select, fused sparse prefill + compaction."""
     from paper_2410_08584_b200 import workloads as W
     res = []
-    for tau in (0.95, 0.99):
+    for tau in taus:
         lay = W.video_layer(tau=tau)
         q, k, v, probe = (t.to(dev) for t in (lay.q, lay.k, lay.v, lay.probe_pos))
         desc = z.layer_desc(q, k)
@@ -327,7 +327,7 @@ def long_video_benchmark(z, dev, peaks, reps=10):
         # the same launch back to back for about half a second: the figure under the power cap,
         # the one to hold against the sustained GEMM peak (the 10-launch figure is a burst)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        n_sust = 250
+        n_sust = max(sustained, 1)
         e0.record()
         for _ in range(n_sust):
             z.zipvl_sparse_prefill(desc, q, k, v, idx, k_dev, lay.L, out=out, ws=ws_pf, status=st)
@@ -600,6 +600,10 @@ def run_ours(args, rank, world, local):
     dev = torch.device("cuda", local)
     peaks = read_peaks()
 
+    if args.only_long_video:
+        if rank == 0:
+            print(json.dumps({"long_video": long_video_benchmark(z, dev, peaks, reps=3, taus=(0.95,), sustained=0)}))
+        return
     seed0 = replicas.replica_seed(BASE_SEED, rank)
     layers = [W.heavy_key_layer(seed=seed0 + s, probe_seed=seed0 + 7919) for s in range(N_SETS)]
     run = LayerRunner(z, layers, dev)
@@ -622,7 +626,7 @@ def run_ours(args, rank, world, local):
     t1e.record()
     torch.cuda.synchronize()
     est_ms = max(t0e.elapsed_time(t1e) / K, 1e-3)
-    repeats = max(1, int(math.ceil(1.1 * MIN_REGION_MS / (est_ms * K))))
+    repeats = max(1, int(math.ceil(1.1 * args.min_region_ms / (est_ms * K))))
     n_ev = min(repeats * K, 400)
     events = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(n_ev)]
     events2 = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(K)]
@@ -656,6 +660,18 @@ def run_ours(args, rank, world, local):
     torch.cuda.synchronize()
     per_call = np.array([[ev[j].elapsed_time(ev[j + 1]) for j in range(5)] for ev in events2])
     call_ms = per_call.mean(axis=0)
+    # the dominant kernel alone, back to back over the rotating inputs (no event between launches,
+    # so each launch's set-up overlaps the one before, as it does inside a step)
+    b0, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n_b2b = 10 * N_SETS
+    b0.record()
+    for i in range(n_b2b):
+        qb, kb_, vb = run.sets[i % N_SETS]
+        z.zipvl_sparse_prefill_compact(run.desc, qb, kb_, vb, run.idx, run.k_dev, run.L, run.kc, run.vc, run.cap,
+                                       out=run.out, len_out=run.seq, ws=run.ws_pf, status=run.status)
+    b1.record()
+    torch.cuda.synchronize()
+    pf_b2b_ms = b0.elapsed_time(b1) / n_b2b
     # one sampled check of the timed configuration, outside the timed region
     run.step(0, fused=True)
     torch.cuda.synchronize()
@@ -739,7 +755,10 @@ def run_ours(args, rank, world, local):
                                   else " (burst bf16: region < 1 s or no power cap seen)"),
             "traffic": traffic.get("bytes_per_launch"), "traffic_unit": "bytes per launch (ncu)",
             "traffic_source": traffic.get("source"),
-            "flops_per_launch": flops, "ms_per_launch": pf_ms}
+            "flops_per_launch": flops, "ms_per_launch": pf_ms,
+            # (context: the same launch back to back, no event records in between)
+            "ms_per_launch_back_to_back": pf_b2b_ms,
+            "frac_burst_back_to_back": flops / (pf_b2b_ms * 1e-3) / 1e12 / peaks["tf_burst"]}
     row_b = hl.n_kv_heads * d * 2
     others = {
         "zipvl_score": {"bound": "hbm", "bytes": L * row_b + 128 * Hq * d * 2 + 8 * L,
@@ -850,6 +869,10 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-long-video", action="store_true", help="skip the long-video (18K-token GQA) leg")
     ap.add_argument("--no-batched", action="store_true", help="skip the 4-sequences-per-call leg")
+    ap.add_argument("--min-region-ms", type=float, default=MIN_REGION_MS,
+                    help="the K-step loop is repeated until the timed region spans this long (0: K steps only, for profiler runs)")
+    ap.add_argument("--only-long-video", action="store_true",
+                    help="run the long-video leg alone and print its record (a light command for profiler captures)")
     ap.add_argument("--library-context", action="store_true",
                     help="also time library attention (flash_attn) on gathered copies and dense, for context")
     ap.add_argument("--stack-layers", type=int, default=40,
