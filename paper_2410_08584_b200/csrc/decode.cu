@@ -350,13 +350,23 @@ zipvl_status run(const zipvl_decode_desc &d, float scale_log2, const void *q, co
     const int n_chunks = (max_len + chunk - 1) / chunk;
     float *wsf = reinterpret_cast<float *>(ws);
     int *lens = reinterpret_cast<int *>(reinterpret_cast<char *>(ws) + partial_bytes(B, Hq, D, max_len));
-#define ZIPVL_DEC(GT_)                                                                          \
+    // Small steps (a request or a few: tens of megabytes) are a matter of latency, and eight
+    // rows in flight per lane group halve the number of dependent load rounds; large batches
+    // stream at the memory's rate either way and run better with the smaller register
+    // footprint of four (more CTAs per SM).
+    const bool deep = (long long)B * Hq * max_len <= (1ll << 20);
+#define ZIPVL_DEC_U(GT_, U_)                                                                    \
     {                                                                                           \
         dim3 grid(n_chunks, Hkv * ((G + GT_ - 1) / GT_), B);                                    \
-        le = launch_dependent(decode_kernel<T, D, GT_, (GT_ <= 2 ? 8 : 4)>, grid, dim3(kDecThreads), 0, st, Hq, Hkv, \
+        le = launch_dependent(decode_kernel<T, D, GT_, U_>, grid, dim3(kDecThreads), 0, st, Hq, Hkv, \
                               scale_log2, (const T *)q, (const T *)k_new, (const T *)v_new,           \
                               (T *)k_cache, (T *)v_cache, cache_off, pg, capacity, seq_lens, max_len, \
                               chunk, n_chunks, wsf, lens, (T *)out, status_word);                    \
+    }
+#define ZIPVL_DEC(GT_)                                                                          \
+    {                                                                                           \
+        if (deep && GT_ <= 2) ZIPVL_DEC_U(GT_, (GT_ <= 2 ? 8 : 4))                              \
+        else ZIPVL_DEC_U(GT_, 4)                                                                \
     }
     cudaError_t le = cudaSuccess;
     if (G == 1) ZIPVL_DEC(1)
@@ -364,6 +374,7 @@ zipvl_status run(const zipvl_decode_desc &d, float scale_log2, const void *q, co
     else if (G <= 4) ZIPVL_DEC(4)
     else ZIPVL_DEC(8)
 #undef ZIPVL_DEC
+#undef ZIPVL_DEC_U
     if (le == cudaSuccess)
         le = launch_dependent(decode_merge_kernel<T, D>, dim3((Hq * D * kMergeLanes + 255) / 256, B), dim3(256), 0, st, Hq,
                               chunk, n_chunks, (const float *)wsf, (const int *)lens, seq_lens, (T *)out);
