@@ -61,7 +61,9 @@ __device__ __forceinline__ void unpack<float, 4>(const uint4 r, float (&x)[4]) {
 }
 
 // kDecUnroll: rows per lane group in flight before any is consumed (8 where the registers allow)
-template <typename T, int D, int GT, int kDecUnroll>
+// kPaged: the cache rows are found through a block table (a separate instantiation, so that the
+// contiguous path carries none of its address arithmetic)
+template <typename T, int D, int GT, int kDecUnroll, bool kPaged>
 __global__ void __launch_bounds__(kDecThreads)
 decode_kernel(int Hq, int Hkv, float scale_log2, const T *__restrict__ q,
               const T *__restrict__ k_new, const T *__restrict__ v_new, T *__restrict__ k_cache,
@@ -109,7 +111,7 @@ decode_kernel(int Hq, int Hkv, float scale_log2, const T *__restrict__ q,
     // zero output) and reported: none of its rows can be trusted to lie inside the cache.
     const int old_len = seq_lens[b];
     const int cap = capacity[b];
-    const long long coff = pg.table ? 0ll : cache_off[b];
+    const long long coff = kPaged ? 0ll : cache_off[b];
     const bool bad = old_len < 0 || old_len > cap || ((coff * (long long)sizeof(T)) & 15) != 0;
     if (bad && first) report(status_word, ZIPVL_DEV_BAD_INDEX);
     const bool appended = !bad && k_new != nullptr && old_len < cap;
@@ -143,9 +145,9 @@ decode_kernel(int Hq, int Hkv, float scale_log2, const T *__restrict__ q,
         T *vb = v_cache + coff + head_off;
         // element offset of a cache row from kb / vb; -1 for a page outside the pool (reported,
         // the row is skipped)
-        const int32_t *my_table = pg.table ? pg.table + (long long)b * pg.stride : nullptr;
+        const int32_t *my_table = kPaged ? pg.table + (long long)b * pg.stride : nullptr;
         auto row_off = [&](int row) -> long long {
-            if (my_table == nullptr) return row * row_pitch;
+            if (!kPaged) return row * row_pitch;
             const int page = my_table[row >> pg.shift];
             if (page < 0 || page >= pg.n_pages) { report(status_word, ZIPVL_DEV_BAD_INDEX); return -1; }
             return (((long long)page << pg.shift) + (row & ((1 << pg.shift) - 1))) * row_pitch;
@@ -350,23 +352,18 @@ zipvl_status run(const zipvl_decode_desc &d, float scale_log2, const void *q, co
     const int n_chunks = (max_len + chunk - 1) / chunk;
     float *wsf = reinterpret_cast<float *>(ws);
     int *lens = reinterpret_cast<int *>(reinterpret_cast<char *>(ws) + partial_bytes(B, Hq, D, max_len));
-    // Small steps (a request or a few: tens of megabytes) are a matter of latency, and eight
-    // rows in flight per lane group halve the number of dependent load rounds; large batches
-    // stream at the memory's rate either way and run better with the smaller register
-    // footprint of four (more CTAs per SM).
-    const bool deep = (long long)B * Hq * max_len <= (1ll << 20);
-#define ZIPVL_DEC_U(GT_, U_)                                                                    \
+#define ZIPVL_DEC_P(GT_, P_)                                                                    \
     {                                                                                           \
         dim3 grid(n_chunks, Hkv * ((G + GT_ - 1) / GT_), B);                                    \
-        le = launch_dependent(decode_kernel<T, D, GT_, U_>, grid, dim3(kDecThreads), 0, st, Hq, Hkv, \
-                              scale_log2, (const T *)q, (const T *)k_new, (const T *)v_new,           \
+        le = launch_dependent(decode_kernel<T, D, GT_, (GT_ <= 2 ? 8 : 4), P_>, grid, dim3(kDecThreads), 0, st, \
+                              Hq, Hkv, scale_log2, (const T *)q, (const T *)k_new, (const T *)v_new,  \
                               (T *)k_cache, (T *)v_cache, cache_off, pg, capacity, seq_lens, max_len, \
                               chunk, n_chunks, wsf, lens, (T *)out, status_word);                    \
     }
 #define ZIPVL_DEC(GT_)                                                                          \
     {                                                                                           \
-        if (deep && GT_ <= 2) ZIPVL_DEC_U(GT_, (GT_ <= 2 ? 8 : 4))                              \
-        else ZIPVL_DEC_U(GT_, 4)                                                                \
+        if (pg.table) ZIPVL_DEC_P(GT_, true)                                                    \
+        else ZIPVL_DEC_P(GT_, false)                                                            \
     }
     cudaError_t le = cudaSuccess;
     if (G == 1) ZIPVL_DEC(1)
@@ -374,7 +371,7 @@ zipvl_status run(const zipvl_decode_desc &d, float scale_log2, const void *q, co
     else if (G <= 4) ZIPVL_DEC(4)
     else ZIPVL_DEC(8)
 #undef ZIPVL_DEC
-#undef ZIPVL_DEC_U
+#undef ZIPVL_DEC_P
     if (le == cudaSuccess)
         le = launch_dependent(decode_merge_kernel<T, D>, dim3((Hq * D * kMergeLanes + 255) / 256, B), dim3(256), 0, st, Hq,
                               chunk, n_chunks, (const float *)wsf, (const int *)lens, seq_lens, (T *)out);
