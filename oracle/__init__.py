@@ -231,3 +231,113 @@ def decode_step_paged(q, k_new, v_new, k_pages, v_pages, block_table, seq_lens, 
                 k_pages[page, r % page_rows] = kc[b, r]
                 v_pages[page, r % page_rows] = vc[b, r]
     return out
+
+
+# ---------------------------------------------------------------------------------------
+# Mixed-precision KV cache (Sec. 4.3, Table 3: "important tokens are quantized to 4-bit,
+# while other tokens are quantized to 2-bit").  The paper takes the quantiser from the work
+# it cites and only fixes the bit allocation; the reading used here: every token stays in
+# the cache; keys and values are quantised per (token, KV head) over the head_dim channels
+# with an asymmetric uniform quantiser whose scale and zero point are kept in the storage
+# type; the codes are decided in fp32 (the precision the kernel takes that decision in).
+# ---------------------------------------------------------------------------------------
+def _round_to_storage(x, storage):
+    """fp32 values rounded (to nearest even) to the storage type, returned as fp32."""
+    import torch
+    t = torch.from_numpy(np.ascontiguousarray(x, np.float32))
+    if storage == "bf16":
+        return t.to(torch.bfloat16).float().numpy()
+    if storage == "f16":
+        return t.to(torch.float16).float().numpy()
+    return t.numpy().copy()
+
+
+def quantize_rows(x, bits, storage="bf16"):
+    """x float32 [n, H, d] (stored values).  Per (row, head): lo = min, hi = max over the d
+    channels, scale = (hi - lo) / (2^bits - 1) in fp32; scale and lo are rounded to the
+    storage type; code_c = clip(rint((x_c - lo) / scale), 0, 2^bits - 1), every step in fp32.
+    A row of equal values (scale 0) gets codes 0.  Returns (codes uint8 [n,H,d],
+    scale float32 [n,H], zero float32 [n,H])."""
+    x = np.ascontiguousarray(x, np.float32)
+    levels = np.float32((1 << bits) - 1)
+    lo = x.min(axis=-1)
+    hi = x.max(axis=-1)
+    scale = _round_to_storage((hi - lo).astype(np.float32) / levels, storage)
+    zero = _round_to_storage(lo, storage)
+    safe = np.where(scale > 0, scale, np.float32(1.0)).astype(np.float32)
+    qf = np.rint(((x - zero[..., None]).astype(np.float32) / safe[..., None]).astype(np.float32))
+    codes = np.clip(qf, 0, levels).astype(np.uint8)
+    codes[scale <= 0] = 0
+    return codes, scale.astype(np.float32), zero.astype(np.float32)
+
+
+def dequantize_rows(codes, scale, zero):
+    """x^ = code * scale + zero, in float64."""
+    return codes.astype(np.float64) * scale.astype(np.float64)[..., None] + zero.astype(np.float64)[..., None]
+
+
+def pack_codes(codes, bits):
+    """Codes of `bits` bits packed little-end first: channel c of a row sits in byte
+    c * bits // 8 at bit offset (c * bits) % 8.  codes uint8 [..., d] -> uint8 [..., d*bits/8]."""
+    codes = np.ascontiguousarray(codes, np.uint8)
+    per = 8 // bits
+    d = codes.shape[-1]
+    assert d % per == 0
+    g = codes.reshape(codes.shape[:-1] + (d // per, per)).astype(np.uint16)
+    out = np.zeros(g.shape[:-1], np.uint16)
+    for i in range(per):
+        out |= g[..., i] << (bits * i)
+    return out.astype(np.uint8)
+
+
+def quantize_kv(K, V, T, storage="bf16", bits_hi=4, bits_lo=2):
+    """The cache of one layer after Algorithm 1 when nothing is evicted but the precision
+    follows the token set: the tokens of T (ascending) at bits_hi bits, the others
+    (ascending) at bits_lo bits.  K, V float32 [L, Hkv, d].  Returns a dict with, for
+    block in ("hi", "lo"): tokens (positions), k_codes, v_codes (uint8 [n,Hkv,d]), k_scale,
+    k_zero, v_scale, v_zero (float32 [n,Hkv])."""
+    K, V = _f32(K), _f32(V)
+    T = np.asarray(T, np.int64)
+    U = np.setdiff1d(np.arange(K.shape[0]), T)
+    cache = {}
+    for name, toks, bits in (("hi", T, bits_hi), ("lo", U, bits_lo)):
+        kc, ks, kz = quantize_rows(K[toks], bits, storage)
+        vc, vs, vz = quantize_rows(V[toks], bits, storage)
+        cache[name] = dict(tokens=toks, bits=bits, k_codes=kc, v_codes=vc, k_scale=ks, k_zero=kz,
+                           v_scale=vs, v_zero=vz)
+    return cache
+
+
+def decode_step_quant(q, k_new, v_new, cache, n_kv_heads, storage="bf16", scale=None):
+    """Algorithm 2 (Eq. 4-5) over the mixed-precision cache of one request: the new key and
+    value (float32 [1,Hkv,d], or None) are quantised at the high precision and appended to
+    the "hi" block (Eq. 4); the query (float32 [1,Hq,d]) attends over the dequantised rows of
+    both blocks (Eq. 5; softmax attention does not depend on the order of the cached rows).
+    The cache dict is updated in place.  Returns float64 [1, Hq, d]."""
+    hi, lo = cache["hi"], cache["lo"]
+    if k_new is not None:
+        kc, ks, kz = quantize_rows(_f32(k_new), hi["bits"], storage)
+        vc, vs, vz = quantize_rows(_f32(v_new), hi["bits"], storage)
+        for key, val in (("k_codes", kc), ("v_codes", vc), ("k_scale", ks), ("k_zero", kz),
+                         ("v_scale", vs), ("v_zero", vz)):
+            hi[key] = np.concatenate([hi[key], val])
+        hi["tokens"] = np.concatenate([hi["tokens"], [-1]])
+    kd = np.concatenate([dequantize_rows(b["k_codes"], b["k_scale"], b["k_zero"]) for b in (hi, lo)])
+    vd = np.concatenate([dequantize_rows(b["v_codes"], b["v_scale"], b["v_zero"]) for b in (hi, lo)])
+    n = kd.shape[0]
+    # the dequantised rows are fp64; decode_step takes float32 caches, so the attention over
+    # them is written out here directly, in float64
+    q = np.asarray(q, np.float64)
+    _, Hq, d = q.shape
+    G = Hq // n_kv_heads
+    sc = default_scale(d) if scale is None else float(scale)
+    out = np.zeros((1, Hq, d), np.float64)
+    for h in range(Hq):
+        g = h // G
+        if n == 0:
+            continue
+        s = sc * (kd[:, g, :] @ q[0, h])
+        w = np.exp(s - s.max())
+        w /= w.sum()
+        out[0, h] = w @ vd[:, g, :]
+    return out

@@ -500,3 +500,81 @@ def test_paged_decode_is_decode_on_the_gathered_rows():
     for b in range(B):
         assert np.array_equal(kp[perm[b, lens[b] // page_rows], lens[b] % page_rows], kn[b])
         assert np.array_equal(vp[perm[b, lens[b] // page_rows], lens[b] % page_rows], vn[b])
+
+
+# ---- mixed-precision KV cache (Sec. 4.3, Table 3): the quantiser reading and its packing ----
+def _grid_rows(rng, n, H, d, bits, zero=-1.5, scale=0.25):
+    """Rows that lie exactly on a quantisation grid whose zero point and scale are exact in
+    bfloat16, with the smallest and the largest code present in every (row, head)."""
+    codes = rng.integers(0, 1 << bits, (n, H, d)).astype(np.uint8)
+    codes[..., 0] = 0
+    codes[..., 1] = (1 << bits) - 1
+    return codes, (zero + scale * codes.astype(np.float32)).astype(np.float32)
+
+
+def test_quantiser_recovers_rows_that_lie_on_its_grid():
+    rng = np.random.default_rng(5)
+    for bits in (4, 2):
+        codes, x = _grid_rows(rng, 7, 3, 32, bits)
+        c, s, z = oracle.quantize_rows(x, bits, "bf16")
+        assert np.array_equal(c, codes) and np.all(s == 0.25) and np.all(z == -1.5)
+        assert np.array_equal(oracle.dequantize_rows(c, s, z), x.astype(np.float64))
+
+
+def test_quantiser_round_trip_error_is_half_a_step_plus_the_parameter_rounding():
+    rng = np.random.default_rng(6)
+    x = (rng.standard_normal((50, 4, 64)) * rng.uniform(0.1, 5.0, (50, 4, 1))).astype(np.float32)
+    for bits in (4, 2):
+        levels = (1 << bits) - 1
+        c, s, z = oracle.quantize_rows(x, bits, "bf16")
+        assert c.max() <= levels
+        err = np.abs(oracle.dequantize_rows(c, s, z) - x)
+        lo, hi = x.min(-1), x.max(-1)
+        slack = np.maximum(0, (hi - z) - levels * s) + np.maximum(0, z - lo)      # what the bf16 parameters miss
+        assert np.all(err <= (0.5 * s + slack)[..., None] * (1 + 1e-6) + 1e-7)
+        # the parameters are the storage type's roundings of min and (max - min) / levels
+        assert np.all(np.abs(z - lo) <= np.abs(lo) * 2.0 ** -8)
+        assert np.all(np.abs(s - (hi - lo) / levels) <= (hi - lo) / levels * 2.0 ** -8)
+        # codes are monotone in the value within a row
+        order = np.argsort(x, axis=-1)
+        assert np.all(np.diff(np.take_along_axis(c.astype(int), order, -1), axis=-1) >= 0)
+
+
+def test_quantiser_constant_row_and_packing():
+    x = np.full((2, 1, 8), 0.75, np.float32)
+    c, s, z = oracle.quantize_rows(x, 4, "bf16")
+    assert not c.any() and np.all(s == 0) and np.all(oracle.dequantize_rows(c, s, z) == 0.75)
+    # bytes written out by hand: 4-bit pairs low nibble first, 2-bit quads lowest bits first
+    assert oracle.pack_codes(np.array([[1, 2, 3, 4, 15, 0, 9, 10]], np.uint8), 4).tolist() == [[0x21, 0x43, 0x0F, 0xA9]]
+    assert oracle.pack_codes(np.array([[1, 2, 3, 0, 3, 3, 3, 3]], np.uint8), 2).tolist() == [[0b00111001, 0xFF]]
+
+
+def test_mixed_precision_cache_split_and_lossless_decode():
+    """Tokens of T at 4 bits in T's order, the rest at 2 bits ascending; on data that both grids
+    hold exactly, a decode step over the quantised cache is the dense decode step over all L
+    rows (softmax attention does not depend on the order of the cached rows), and the appended
+    token joins the 4-bit block."""
+    rng = np.random.default_rng(7)
+    L, Hq, Hkv, d = 40, 4, 2, 16
+    T = np.sort(rng.choice(L, 13, replace=False))
+    U = np.setdiff1d(np.arange(L), T)
+    K = np.zeros((L, Hkv, d), np.float32)
+    V = np.zeros((L, Hkv, d), np.float32)
+    for toks, bits in ((T, 4), (U, 2)):
+        K[toks] = _grid_rows(rng, len(toks), Hkv, d, bits)[1]
+        V[toks] = _grid_rows(rng, len(toks), Hkv, d, bits, zero=0.5, scale=0.125)[1]
+    cache = oracle.quantize_kv(K, V, T, "bf16")
+    assert np.array_equal(cache["hi"]["tokens"], T) and np.array_equal(cache["lo"]["tokens"], U)
+    assert cache["hi"]["k_codes"].max() <= 15 and cache["lo"]["k_codes"].max() <= 3
+    q = rng.standard_normal((1, Hq, d)).astype(np.float32)
+    kn = _grid_rows(rng, 1, Hkv, d, 4)[1]
+    vn = _grid_rows(rng, 1, Hkv, d, 4, zero=0.5, scale=0.125)[1]
+    got = oracle.decode_step_quant(q, kn, vn, cache, Hkv)
+    kc = np.concatenate([K, np.zeros((1, Hkv, d), np.float32)]).reshape(-1)
+    vc = np.concatenate([V, np.zeros((1, Hkv, d), np.float32)]).reshape(-1)
+    seq = np.array([L], np.int32)
+    want = oracle.decode_step(q, kn, vn, kc, vc, np.zeros(1, np.int64), seq, Hkv)
+    assert np.abs(got - want).max() < 1e-12
+    assert len(cache["hi"]["tokens"]) == len(T) + 1 and len(cache["lo"]["tokens"]) == len(U)
+    assert np.array_equal(oracle.dequantize_rows(cache["hi"]["k_codes"][-1:], cache["hi"]["k_scale"][-1:],
+                                                 cache["hi"]["k_zero"][-1:]), kn.astype(np.float64))
