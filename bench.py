@@ -504,6 +504,67 @@ def batched_benchmark(z, dev, layers, peaks, n_seq=4, reps=40):
             "note": "score + select + sparse prefill with compaction for 4 sequences per call (no decode step)"}
 
 
+def quant_benchmark(z, dev, layer, peaks, reps=50):
+    """The mixed-precision cache on the benchmark's layer (Table 3's setting: tokens of T at 4 bits,
+    the others at 2, nothing evicted): time to build it, time of a decode step over it (replayed from
+    a CUDA graph: the step is three small launches), its size against the 16-bit cache, and one step
+    checked against the oracle."""
+    import oracle
+    q, k, v, probe = (t.to(dev) for t in (layer.q, layer.k, layer.v, layer.probe_pos))
+    L, Hq, Hkv, d = layer.L, layer.n_q_heads, layer.n_kv_heads, layer.head_dim
+    desc = z.layer_desc(q, k)
+    st = torch.zeros(1, dtype=torch.int32, device=dev)
+    acc, norm = z.zipvl_score(desc, q, k, probe)
+    k_dev, idx = z.zipvl_select(acc, norm, layer.tau)
+    kk = int(k_dev.item())
+    caches = [z.QuantCache(L, Hkv, d, torch.bfloat16, dev, cap_hi=kk + 8, cap_lo=L - kk + 1) for _ in range(6)]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    def graph_ms(fn):
+        """fn(cache) for each of the caches, captured once and replayed: per-call GPU time (the
+        calls are short enough that a Python loop would time the host)."""
+        side = torch.cuda.Stream(device=dev)
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            fn(caches[0])
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=side):
+                for c in caches:
+                    fn(c)
+        torch.cuda.current_stream().wait_stream(side)
+        graph.replay()
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(reps):
+            graph.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / (reps * len(caches))
+
+    t_quant = graph_ms(lambda c: z.zipvl_quantize_kv(desc, k, v, idx, k_dev, L, c, status=st))
+    ddesc = z.zipvl_decode_desc(1, Hq, Hkv, d, z.ZIPVL_BF16, 0.0)
+    g = torch.Generator().manual_seed(79)
+    qn = torch.randn(1, Hq, d, generator=g).bfloat16()
+    out = torch.empty(1, Hq, d, dtype=torch.bfloat16, device=dev)
+    lay = z.zipvl_layer(L + 8, Hq, Hkv, d, z.ZIPVL_BF16, 0, 0, 0, 0.0, 0)
+    ws = z.workspace(z.zipvl_workspace_bytes(z.OP_DECODE, lay, 0, 1), dev)
+    qd = qn.to(dev)
+    t_dec = graph_ms(lambda c: z.zipvl_decode_quant(ddesc, qd, None, None, c, L + 8, out=out, ws=ws, status=st))
+    f = lambda t: t.float().cpu().numpy()
+    ref = oracle.quantize_kv(f(layer.k), f(layer.v), idx[:kk].cpu().numpy(), "bf16")
+    want = oracle.decode_step_quant(f(qn), None, None, ref, Hkv, "bf16")
+    dd = np.abs(f(out).astype(np.float64) - want)
+    nbytes = caches[0].nbytes(kk, L - kk)
+    return {"k": kk, "L": L, "quantize_ms": t_quant, "decode_step_ms": t_dec,
+            "cache_bytes": int(nbytes), "cache_bytes_16bit_all_tokens": int(4 * L * Hkv * d),
+            "cache_bytes_16bit_kept_tokens": int(4 * kk * Hkv * d),
+            "compression_vs_16bit_all_tokens": 4.0 * L * Hkv * d / nbytes,
+            "decode_gbs": nbytes / (t_dec * 1e-3) / 1e9, "frac_of_hbm_peak": nbytes / (t_dec * 1e-3) / 1e9 / peaks["hbm"],
+            "device_status_word": int(st.item()),
+            "check": {"checked": bool(dd.max() <= 2e-2 and dd.mean() <= 2e-3), "max_abs": float(dd.max()),
+                      "mean_abs": float(dd.mean())},
+            "note": "both calls timed per call inside a CUDA-graph replay over 6 caches; no token evicted"}
+
+
 def decode_benchmark(z, dev, steps, peaks, B=16, ctx_max=32768):
     """Batched decode on compacted caches (16 requests, contexts 4K-32K, 32 heads
     x 128, bf16) against the same kernel on the uncompacted caches."""
@@ -787,6 +848,13 @@ def run_ours(args, rank, world, local):
         except Exception as e:  # report, never hide
             batched = {"error": repr(e)}
 
+    quant = None
+    if not args.no_batched:
+        try:
+            quant = quant_benchmark(z, dev, layers[0], peaks)
+        except Exception as e:  # report, never hide
+            quant = {"error": repr(e)}
+
     stack = None
     if args.stack_layers > 0:
         try:
@@ -845,7 +913,7 @@ def run_ours(args, rank, world, local):
         "graph_replay_ms_per_step": graph_ms,
         "prefill_ms": float(call_ms[0] + call_ms[1] + call_ms[2]),
         "prefill_tflops_selected": flops / (float(call_ms[0] + call_ms[1] + call_ms[2]) * 1e-3) / 1e12,
-        "roofline": roof, "other_kernels": others, "decode": dec, "batched": batched, "stack": stack, "long_video": video, "library_context": context,
+        "roofline": roof, "other_kernels": others, "decode": dec, "batched": batched, "kv_quant": quant, "stack": stack, "long_video": video, "library_context": context,
         "cpu_baseline": cpu,
         "e2e": {"value": e2e_ms / world, "unit": "ms", "h2d_bytes_per_step": int(h2d),
                 "d2h_bytes_per_step": int(d2h),

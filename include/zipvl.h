@@ -324,6 +324,40 @@ zipvl_status zipvl_decode_paged(const zipvl_decode_desc *desc, const void *q, co
                                 size_t ws_bytes, int32_t *status_word, void *stream);
 
 /*
+ * zipvl_quantize_kv, zipvl_decode_quant -- the mixed-precision KV cache.
+ * Paper: Sec. 4.3 / Table 3 (the adaptive token set drives a mixed-precision cache: "important
+ * tokens are quantized to 4-bit, while other tokens are quantized to 2-bit"); decode as
+ * Algorithm 2, Eq. 4-5.  The paper takes the quantiser from the work it cites; the reading
+ * built here: no token is evicted; keys and values are quantised per (token, KV head) over the
+ * head_dim channels, scale = (max - min) / (2^b - 1), code = clip(rint((x - min) * (1 / scale)),
+ * 0, 2^b - 1), with scale and min rounded to the storage type and kept beside the codes (each step
+ * a correctly rounded fp32 operation).  The cache of a sequence is two blocks -- softmax
+ * attention does not depend on the order of the cached rows:
+ *   "hi": the tokens of T in T's order at 4 bits; k_hi, v_hi: [cap_hi, Hkv, d/2] bytes,
+ *         params_hi: [cap_hi, Hkv, 4] storage-type values (k scale, k min, v scale, v min);
+ *   "lo": the other tokens, ascending, at 2 bits; k_lo, v_lo: [cap_lo, Hkv, d/4] bytes, params_lo alike.
+ *   Channel c of a row sits in byte c*b/8 at bit (c*b)%8.  lens: device int32[2] = rows in hi, lo.
+ * zipvl_quantize_kv builds the blocks from K, V and the token set (idx ascending, k_dev on the
+ * device, k_max the host's bound) and writes lens_out; a block that is too small is filled to
+ * its capacity and ZIPVL_DEV_CAPACITY reported.  zipvl_decode_quant is one decode step of ONE
+ * request (desc->batch == 1): if k_new != NULL the new key / value ([Hkv,d]) are quantised at
+ * 4 bits and appended to the hi block (lens[0] += 1; a full block: ZIPVL_DEV_CAPACITY, no
+ * append); out[h,:] = softmax attention of q[h,:] over all dequantised rows.  max_len: host
+ * bound on lens[0] + lens[1] after the append; ws: zipvl_workspace_bytes(ZIPVL_OP_DECODE) for
+ * batch 1 and L = max_len.  16-bit storage types, head_dim 64 or 128, 1, 2 or 4 query heads per
+ * KV head, at most 64 KV heads.  The call enqueues two kernels (three with an append).
+ */
+zipvl_status zipvl_quantize_kv(const zipvl_layer *layer, const void *k, const void *v, const int32_t *idx,
+                               const int32_t *k_dev, int32_t k_max, void *k_hi, void *v_hi,
+                               void *params_hi, int32_t cap_hi, void *k_lo, void *v_lo, void *params_lo,
+                               int32_t cap_lo, int32_t *lens_out, int32_t *status_word, void *stream);
+zipvl_status zipvl_decode_quant(const zipvl_decode_desc *desc, const void *q, const void *k_new,
+                                const void *v_new, void *k_hi, void *v_hi, void *params_hi, int32_t cap_hi,
+                                void *k_lo, void *v_lo, void *params_lo, int32_t cap_lo, int32_t *lens,
+                                int32_t max_len, void *out, void *ws, size_t ws_bytes,
+                                int32_t *status_word, void *stream);
+
+/*
  * zipvl_decode_noalloc -- zipvl_decode for callers that cannot allocate.
  * (The paper has no counterpart: this is a deployment variant of the decode
  * step, same arithmetic, same kernels.)

@@ -255,7 +255,8 @@ def _round_to_storage(x, storage):
 def quantize_rows(x, bits, storage="bf16"):
     """x float32 [n, H, d] (stored values).  Per (row, head): lo = min, hi = max over the d
     channels, scale = (hi - lo) / (2^bits - 1) in fp32; scale and lo are rounded to the
-    storage type; code_c = clip(rint((x_c - lo) / scale), 0, 2^bits - 1), every step in fp32.
+    storage type; inv = 1 / scale; code_c = clip(rint((x_c - lo) * inv), 0, 2^bits - 1), every
+    step one fp32 operation (one division per row, a subtraction and a multiplication per value).
     A row of equal values (scale 0) gets codes 0.  Returns (codes uint8 [n,H,d],
     scale float32 [n,H], zero float32 [n,H])."""
     x = np.ascontiguousarray(x, np.float32)
@@ -265,7 +266,8 @@ def quantize_rows(x, bits, storage="bf16"):
     scale = _round_to_storage((hi - lo).astype(np.float32) / levels, storage)
     zero = _round_to_storage(lo, storage)
     safe = np.where(scale > 0, scale, np.float32(1.0)).astype(np.float32)
-    qf = np.rint(((x - zero[..., None]).astype(np.float32) / safe[..., None]).astype(np.float32))
+    inv = (np.float32(1.0) / safe).astype(np.float32)
+    qf = np.rint(((x - zero[..., None]).astype(np.float32) * inv[..., None]).astype(np.float32))
     codes = np.clip(qf, 0, levels).astype(np.uint8)
     codes[scale <= 0] = 0
     return codes, scale.astype(np.float32), zero.astype(np.float32)

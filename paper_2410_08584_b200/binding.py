@@ -26,7 +26,7 @@ EXPORTS = ["zipvl_status_string", "zipvl_last_error", "zipvl_version", "zipvl_la
            "zipvl_score", "zipvl_select", "zipvl_sparse_prefill", "zipvl_compact_kv",
            "zipvl_sparse_prefill_compact", "zipvl_workspace_bytes_batch", "zipvl_score_batch",
            "zipvl_select_batch", "zipvl_sparse_prefill_batch",
-           "zipvl_decode", "zipvl_decode_paged", "zipvl_decode_noalloc", "zipvl_prefill_layer_host", "zipvl_layer_step_host",
+           "zipvl_decode", "zipvl_decode_paged", "zipvl_quantize_kv", "zipvl_decode_quant", "zipvl_decode_noalloc", "zipvl_prefill_layer_host", "zipvl_layer_step_host",
            "zipvl_release_host_scratch", "zipvl_selftest_wait_timeout"]
 
 
@@ -103,6 +103,11 @@ def load():
     lib.zipvl_decode_paged.restype = C.c_int
     lib.zipvl_decode_paged.argtypes = [C.POINTER(zipvl_decode_desc), vp, vp, vp, vp, vp, vp, i32, i32, i32,
                                        vp, vp, i32, vp, vp, sz, vp, vp]
+    lib.zipvl_quantize_kv.restype = C.c_int
+    lib.zipvl_quantize_kv.argtypes = [lp, vp, vp, vp, vp, i32, vp, vp, vp, i32, vp, vp, vp, i32, vp, vp, vp]
+    lib.zipvl_decode_quant.restype = C.c_int
+    lib.zipvl_decode_quant.argtypes = [C.POINTER(zipvl_decode_desc), vp, vp, vp, vp, vp, vp, i32, vp, vp, vp, i32,
+                                       vp, i32, vp, vp, sz, vp, vp]
     lib.zipvl_decode_noalloc.restype = C.c_int
     lib.zipvl_decode_noalloc.argtypes = [C.POINTER(zipvl_decode_desc), vp, vp, vp, vp, vp, vp, vp,
                                          vp, i32, vp, vp, vp]
@@ -368,6 +373,56 @@ def zipvl_decode_paged(desc, q, k_new, v_new, k_pages, v_pages, block_table, cap
     _check(load().zipvl_decode_paged(C.byref(desc), _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(k_pages),
                                      _ptr(v_pages), _ptr(block_table), block_table.shape[1],
                                      k_pages.shape[1], k_pages.shape[0], _ptr(capacity), _ptr(seq_lens),
+                                     int(max_len), _ptr(out), _ptr(ws), ws.numel(), _ptr(status),
+                                     _stream(stream)))
+    return out
+
+
+class QuantCache:
+    """Device buffers of one sequence's mixed-precision cache (see zipvl_quantize_kv in
+    include/zipvl.h): 4-bit block for the tokens of T plus room for `extra` decoded tokens,
+    2-bit block for the others."""
+
+    def __init__(self, L, n_kv_heads, head_dim, dtype, device, cap_hi, cap_lo):
+        u8 = torch.uint8
+        self.cap_hi, self.cap_lo = int(cap_hi), int(cap_lo)
+        self.k_hi = torch.zeros(self.cap_hi, n_kv_heads, head_dim // 2, dtype=u8, device=device)
+        self.v_hi = torch.zeros_like(self.k_hi)
+        self.p_hi = torch.zeros(self.cap_hi, n_kv_heads, 4, dtype=dtype, device=device)
+        self.k_lo = torch.zeros(self.cap_lo, n_kv_heads, head_dim // 4, dtype=u8, device=device)
+        self.v_lo = torch.zeros_like(self.k_lo)
+        self.p_lo = torch.zeros(self.cap_lo, n_kv_heads, 4, dtype=dtype, device=device)
+        self.lens = torch.zeros(2, dtype=torch.int32, device=device)
+
+    def nbytes(self, n_hi, n_lo):
+        """Bytes the first n_hi / n_lo rows of the blocks take (codes of K and V + parameters)."""
+        per_hi = 2 * self.k_hi[0].numel() + self.p_hi[0].numel() * self.p_hi.element_size()
+        per_lo = 2 * self.k_lo[0].numel() + self.p_lo[0].numel() * self.p_lo.element_size()
+        return n_hi * per_hi + n_lo * per_lo
+
+
+def zipvl_quantize_kv(layer, k, v, idx, k_dev, k_max, cache, status=None, stream=None):
+    """K, V and the token set into the mixed-precision cache; returns cache.lens (device int32[2])."""
+    _dev(k, "k", token_strided=True), _dev(v, "v", token_strided=True), _dev(idx, "idx", torch.int32)
+    _same_stride(k, v)
+    _check(load().zipvl_quantize_kv(C.byref(layer), _ptr(k), _ptr(v), _ptr(idx), _ptr(k_dev), int(k_max),
+                                    _ptr(cache.k_hi), _ptr(cache.v_hi), _ptr(cache.p_hi), cache.cap_hi,
+                                    _ptr(cache.k_lo), _ptr(cache.v_lo), _ptr(cache.p_lo), cache.cap_lo,
+                                    _ptr(cache.lens), _ptr(status), _stream(stream)))
+    return cache.lens
+
+
+def zipvl_decode_quant(desc, q, k_new, v_new, cache, max_len, out=None, ws=None, status=None, stream=None):
+    """One decode step of one request over its mixed-precision cache; returns out [1,Hq,d]."""
+    _dev(q, "q")
+    out = torch.empty_like(q) if out is None else out
+    if ws is None:
+        lay = zipvl_layer(int(max_len), desc.n_q_heads, desc.n_kv_heads, desc.head_dim, desc.dtype,
+                          0, 0, 0, 0.0, 0)
+        ws = workspace(zipvl_workspace_bytes(OP_DECODE, lay, 0, 1), q.device)
+    _check(load().zipvl_decode_quant(C.byref(desc), _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(cache.k_hi),
+                                     _ptr(cache.v_hi), _ptr(cache.p_hi), cache.cap_hi, _ptr(cache.k_lo),
+                                     _ptr(cache.v_lo), _ptr(cache.p_lo), cache.cap_lo, _ptr(cache.lens),
                                      int(max_len), _ptr(out), _ptr(ws), ws.numel(), _ptr(status),
                                      _stream(stream)))
     return out

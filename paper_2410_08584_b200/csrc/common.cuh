@@ -144,6 +144,10 @@ zipvl_status launch_compact(const LayerArgs &a, int elem_bytes, const void *k, c
                             cudaStream_t st);
 
 size_t decode_ws_bytes(int B, int Hq, int D, int max_len);
+int decode_chunk_rows(int B, int Hq, int max_len);
+size_t decode_partial_bytes(int B, int Hq, int D, int max_len);
+zipvl_status launch_decode_merge(int dtype, int D, int Hq, int B, int chunk, int n_chunks, const float *ws,
+                                 const int *lens, int32_t *seq_lens, void *out, cudaStream_t st);
 zipvl_status launch_decode(const zipvl_decode_desc &d, float scale_log2, const void *q,
                            const void *k_new, const void *v_new, void *k_cache, void *v_cache,
                            const int64_t *cache_off, const int32_t *capacity, int32_t *seq_lens,

@@ -382,6 +382,26 @@ zipvl_status run(const zipvl_decode_desc &d, float scale_log2, const void *q, co
 
 }  // namespace
 
+// what the decode over a quantised cache (kvquant.cu) shares with this file: the chunking, the
+// layout of the partial results and the merge kernel
+int decode_chunk_rows(int B, int Hq, int max_len) { return decode_chunk(B, Hq, max_len); }
+size_t decode_partial_bytes(int B, int Hq, int D, int max_len) { return partial_bytes(B, Hq, D, max_len); }
+zipvl_status launch_decode_merge(int dtype, int D, int Hq, int B, int chunk, int n_chunks, const float *ws,
+                                 const int *lens, int32_t *seq_lens, void *out, cudaStream_t st) {
+    cudaError_t le = cudaErrorInvalidValue;
+    const dim3 grid((Hq * D * kMergeLanes + 255) / 256, B);
+#define ZIPVL_MERGE(T_, D_) \
+    le = launch_dependent(decode_merge_kernel<T_, D_>, grid, dim3(256), 0, st, Hq, chunk, n_chunks, ws, lens, seq_lens, (T_ *)out)
+    if (dtype == ZIPVL_BF16 && D == 128) ZIPVL_MERGE(__nv_bfloat16, 128);
+    else if (dtype == ZIPVL_BF16 && D == 64) ZIPVL_MERGE(__nv_bfloat16, 64);
+    else if (dtype == ZIPVL_F16 && D == 128) ZIPVL_MERGE(__half, 128);
+    else if (dtype == ZIPVL_F16 && D == 64) ZIPVL_MERGE(__half, 64);
+#undef ZIPVL_MERGE
+    if (le != cudaSuccess) return fail(ZIPVL_ERR_CUDA, "decode merge: launch: %s", cudaGetErrorString(le));
+    count_launches(1);
+    return ZIPVL_OK;
+}
+
 size_t decode_ws_bytes(int B, int Hq, int D, int max_len) {
     return partial_bytes(B, Hq, D, max_len) + counter_bytes(B, Hq);
 }

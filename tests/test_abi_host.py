@@ -117,6 +117,21 @@ def test_argument_validation_without_a_device(lib):
     big = z.zipvl_decode_desc(16, 32, 32, 128, 0, 0.0)
     rc, text = status(lambda: na(C.byref(big), p, None, None, p, p, p, p, p, 32768, p, None, None))
     assert rc == 3 and "scratch" in text
+    # the mixed-precision cache: storage type, head grouping, batch, NULL blocks
+    lay16 = z.zipvl_layer(128, 4, 2, 64, z.ZIPVL_BF16, 0, 0, 0, 0.0, 0)
+    lay32 = z.zipvl_layer(128, 4, 2, 64, z.ZIPVL_F32, 0, 0, 0, 0.0, 0)
+    qk = lib.zipvl_quantize_kv
+    assert qk(C.byref(lay32), p, p, p, p, 128, p, p, p, 8, p, p, p, 8, p, None, None) == 2
+    assert qk(C.byref(lay16), p, p, p, p, 0, p, p, p, 8, p, p, p, 8, p, None, None) == 1
+    assert qk(C.byref(lay16), p, p, p, p, 128, null, p, p, 8, p, p, p, 8, p, None, None) == 1
+    assert qk(C.byref(lay16), p, p, p, p, 128, p, p, p, 0, p, p, p, 8, p, None, None) == 1
+    dq = lib.zipvl_decode_quant
+    d1 = z.zipvl_decode_desc(1, 4, 2, 64, 0, 0.0)
+    assert dq(C.byref(d), p, None, None, p, p, p, 8, p, p, p, 8, p, 16, p, p, 1 << 20, None, None) == 2   # batch 2
+    assert dq(C.byref(d1), p, p, None, p, p, p, 8, p, p, p, 8, p, 16, p, p, 1 << 20, None, None) == 1
+    assert dq(C.byref(d1), p, None, None, p, p, p, 8, p, p, p, 8, p, 16, p, p, 8, None, None) == 3
+    d3 = z.zipvl_decode_desc(1, 6, 2, 64, 0, 0.0)
+    assert dq(C.byref(d3), p, None, None, p, p, p, 8, p, p, p, 8, p, 16, p, p, 1 << 20, None, None) == 2  # 3 heads per KV head
     # the wait self-test: limits outside [1, 2^20] and a missing status word are refused
     assert lib.zipvl_selftest_wait_timeout(0, None, p, None) == 1
     assert lib.zipvl_selftest_wait_timeout(1 << 21, None, p, None) == 1

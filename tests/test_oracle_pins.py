@@ -531,7 +531,7 @@ def test_quantiser_round_trip_error_is_half_a_step_plus_the_parameter_rounding()
         err = np.abs(oracle.dequantize_rows(c, s, z) - x)
         lo, hi = x.min(-1), x.max(-1)
         slack = np.maximum(0, (hi - z) - levels * s) + np.maximum(0, z - lo)      # what the bf16 parameters miss
-        assert np.all(err <= (0.5 * s + slack)[..., None] * (1 + 1e-6) + 1e-7)
+        assert np.all(err <= (0.5 * s + slack)[..., None] * (1 + 1e-5) + 1e-7)
         # the parameters are the storage type's roundings of min and (max - min) / levels
         assert np.all(np.abs(z - lo) <= np.abs(lo) * 2.0 ** -8)
         assert np.all(np.abs(s - (hi - lo) / levels) <= (hi - lo) / levels * 2.0 ** -8)
