@@ -650,7 +650,11 @@ struct SoloCtl {                       // static shared memory
     unsigned long long wsum[kSoloWarps], sum_gt, bin_sum;
     unsigned int wcnt[kSoloWarps], wmin[2][kSoloWarps], wmax[2][kSoloWarps];
     unsigned int hit, hit_bin, cnt_gt, bin_cnt, one_key;
+    // the tokens of a sparsely filled crossing bin, resolved by one warp (see kDirect)
+    unsigned int n_cand, cand_key[32];
+    unsigned long long cand_fx[32];
 };
+constexpr unsigned int kDirect = 32;   // a crossing bin with this many tokens or fewer skips the next level
 
 // block-wide (256 threads) exclusive prefix of a (count, sum) pair in thread order, and totals
 __device__ __forceinline__ void solo_scan(unsigned int vc, unsigned long long vs, SoloCtl &c,
@@ -919,14 +923,54 @@ select_solo_kernel(int L, const float *__restrict__ acc, const float *__restrict
             solo_find_bin(sm, by_sum, target, carry_c, carry_s, c);
             if (c.hit == 0xffffffffu) { found = false; break; }     // (rounding let no prefix qualify)
             if (shift == 0) { thr_key = base + c.hit_bin; break; }  // the bin is one key value
-            if (c.bin_cnt == 1) {
-                // one token: its owner says which key it is
+            if (c.bin_cnt <= kDirect) {
+                // A handful of tokens in the crossing bin: their owners put them on a list and one
+                // warp ranks them against each other -- lane i counts (and sums) the entries above
+                // its own; the threshold is the largest key at which the running total, the copies
+                // of that key included, reaches the target.  This replaces a whole histogram level.
+                const unsigned int above_c = c.cnt_gt;
+                const unsigned long long above_s = c.sum_gt;
+                if (threadIdx.x == 0) c.n_cand = 0;
+                __syncthreads();
 #pragma unroll
                 for (int e = 0; e < kSoloPer; ++e) {
                     unsigned int d;
                     const bool in = (level == 0) ? (d = (keys[e] - base) >> shift, true)
                                                  : solo_bin(keys[e], base, width_log2, shift, &d);
-                    if (j0 + e < L && in && d == c.hit_bin) c.one_key = keys[e];
+                    if (j0 + e < L && in && d == c.hit_bin) {
+                        const unsigned int slot = atomicAdd(&c.n_cand, 1u);
+                        if (slot < kDirect) {
+                            c.cand_key[slot] = keys[e];
+                            c.cand_fx[slot] = by_sum ? to_fx(bud_is_norm ? nv[e] : av[e]) : 0ull;
+                        }
+                    }
+                }
+                __syncthreads();
+                if (threadIdx.x < 32) {
+                    const unsigned int n = min(c.n_cand, kDirect);
+                    const bool mine = (unsigned int)lane < n;
+                    const unsigned int my_key = mine ? c.cand_key[lane] : 0u;
+                    const unsigned long long my_fx = mine ? c.cand_fx[lane] : 0ull;
+                    unsigned int gt_c = 0, eq_c = 0;
+                    unsigned long long gt_s = 0;
+                    for (unsigned int o = 0; o < n; ++o) {
+                        const unsigned int ko = __shfl_sync(0xffffffffu, my_key, o);
+                        const unsigned long long fo = __shfl_sync(0xffffffffu, my_fx, o);
+                        if (ko > my_key) { ++gt_c; gt_s += fo; }
+                        eq_c += (ko == my_key);
+                    }
+                    const unsigned long long eq_s = my_fx * eq_c;
+                    bool hit;
+                    if (by_sum) hit = (above_s + gt_s + eq_s >= target) && (gt_c == 0 || above_s + gt_s < target);
+                    else hit = ((unsigned long long)above_c + gt_c + eq_c >= target) &&
+                               (gt_c == 0 || (unsigned long long)above_c + gt_c < target);
+                    if (mine && hit) {                          // (copies of one key write the same values)
+                        c.cnt_gt = above_c + gt_c;
+                        c.sum_gt = above_s + gt_s;
+                        c.bin_cnt = eq_c;
+                        c.bin_sum = eq_s;
+                        c.one_key = my_key;
+                    }
                 }
                 __syncthreads();
                 thr_key = c.one_key;
