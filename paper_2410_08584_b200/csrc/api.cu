@@ -235,8 +235,9 @@ zipvl_status zipvl_decode(const zipvl_decode_desc *d, const void *q, const void 
         return fail(ZIPVL_ERR_UNSUPPORTED, "zipvl_decode: dtype %d", d->dtype);
     if (d->head_dim != 64 && d->head_dim != 128)
         return fail(ZIPVL_ERR_UNSUPPORTED, "zipvl_decode: head_dim %d (64 or 128)", d->head_dim);
-    if (d->n_q_heads / d->n_kv_heads > 8)
-        return fail(ZIPVL_ERR_UNSUPPORTED, "zipvl_decode: more than 8 query heads per kv head");
+    if (d->n_q_heads / d->n_kv_heads > 8 && !decode_tc_supported(*d))
+        return fail(ZIPVL_ERR_UNSUPPORTED, "zipvl_decode: more than 8 query heads per kv head (up to 32 "
+                                           "in 16-bit storage at head_dim 128)");
     if (!q || !k_cache || !v_cache || !cache_off || !capacity || !seq_lens || !out || !ws)
         return fail(ZIPVL_ERR_INVALID_ARG, "zipvl_decode: NULL pointer");
     if ((k_new == NULL) != (v_new == NULL))

@@ -143,11 +143,27 @@ zipvl_status launch_compact(const LayerArgs &a, int elem_bytes, const void *k, c
                             void *v_cache, int capacity, int32_t *len_out, int32_t *status_word,
                             cudaStream_t st);
 
+// Paged cache: request b's row r lives in page table[b * stride + (r >> shift)] of a pool of
+// n_pages pages of (1 << shift) rows each.  table == nullptr: contiguous caches at cache_off.
+struct PageArgs {
+    const int32_t *table;
+    int stride, shift, n_pages;
+};
+
 size_t decode_ws_bytes(int B, int Hq, int D, int max_len);
 int decode_chunk_rows(int B, int Hq, int max_len);
 size_t decode_partial_bytes(int B, int Hq, int D, int max_len);
 zipvl_status launch_decode_merge(int dtype, int D, int Hq, int B, int chunk, int n_chunks, const float *ws,
                                  const int *lens, int32_t *seq_lens, void *out, cudaStream_t st);
+// Grouped-query decode on the tensor cores (decode_tc.cu): 16-bit storage, head_dim 128, 2 to 32
+// query heads per kv head.  Leaves per-chunk partials and the (length, appended) pairs in the
+// layout of the kernels in decode.cu and returns the chunk it used; the caller launches the merge.
+bool decode_tc_supported(const zipvl_decode_desc &d);
+zipvl_status launch_decode_tc(const zipvl_decode_desc &d, float scale_log2, const void *q,
+                              const void *k_new, const void *v_new, void *k_cache, void *v_cache,
+                              const int64_t *cache_off, PageArgs pg, const int32_t *capacity,
+                              int32_t *seq_lens, int max_len, int min_chunk, float *partials, int *lens,
+                              int32_t *status_word, cudaStream_t st, int *chunk_out);
 zipvl_status launch_decode(const zipvl_decode_desc &d, float scale_log2, const void *q,
                            const void *k_new, const void *v_new, void *k_cache, void *v_cache,
                            const int64_t *cache_off, const int32_t *capacity, int32_t *seq_lens,

@@ -16,6 +16,8 @@
 //   reads the step's length from the workspace, where the first kernel left it.
 // Lengths live on the device; the host only supplies an upper bound.
 #include <math.h>
+#include <stdlib.h>
+#include <string.h>
 
 #include "common.cuh"
 
@@ -23,13 +25,6 @@ namespace zipvl {
 namespace {
 
 constexpr int kDecThreads = 128;
-
-// Paged cache: request b's row r lives in page table[b * stride + (r >> shift)] of a pool of
-// n_pages pages of (1 << shift) rows each.  table == nullptr: contiguous caches at cache_off.
-struct PageArgs {
-    const int32_t *table;
-    int stride, shift, n_pages;
-};
 
 __device__ __forceinline__ uint4 ld_stream(const void *p) {
     uint4 r;
@@ -412,6 +407,30 @@ zipvl_status dispatch_decode(const zipvl_decode_desc &d, float scale_log2, const
                              const int64_t *cache_off, PageArgs pg, const int32_t *capacity,
                              int32_t *seq_lens, int max_len, void *out, void *ws,
                              int32_t *status_word, cudaStream_t st) {
+    // Grouped-query attention in 16-bit storage at head_dim 128 runs on the tensor cores from
+    // three query heads per kv head on: there the CUDA-core kernel is bound by its multiply-adds
+    // (0.51 of the HBM copy rate at four heads per kv head, 0.27 at seven, against 0.76 here;
+    // at two it still reaches 0.81).  ZIPVL_DECODE_KERNEL=simt|tc overrides the choice
+    // (measurements, tests).
+    {
+        const char *env = getenv("ZIPVL_DECODE_KERNEL");
+        const int G = d.n_q_heads / d.n_kv_heads;
+        const bool want_tc = env ? !strcmp(env, "tc") : G >= 3;
+        if (decode_tc_supported(d) && (want_tc || G > 8)) {
+            const int B = d.batch, Hq = d.n_q_heads, D = d.head_dim;
+            float *wsf = reinterpret_cast<float *>(ws);
+            int *lens = reinterpret_cast<int *>(reinterpret_cast<char *>(ws) + partial_bytes(B, Hq, D, max_len));
+            int chunk = 0;
+            const zipvl_status s = launch_decode_tc(d, scale_log2, q, k_new, v_new, k_cache, v_cache, cache_off,
+                                                    pg, capacity, seq_lens, max_len, decode_chunk(B, Hq, max_len),
+                                                    wsf, lens, status_word, st, &chunk);
+            if (s != ZIPVL_OK) return s;
+            const zipvl_status sm = launch_decode_merge(d.dtype, D, Hq, B, chunk, (max_len + chunk - 1) / chunk,
+                                                        wsf, lens, seq_lens, out, st);
+            return sm != ZIPVL_OK ? sm : check_launch("zipvl_decode");
+        }
+        if (G > 8) return fail(ZIPVL_ERR_UNSUPPORTED, "decode: %d query heads per kv head", G);
+    }
 #define ZIPVL_ARGS d, scale_log2, q, k_new, v_new, k_cache, v_cache, cache_off, pg, capacity, \
                    seq_lens, max_len, out, ws, status_word, st
     if (d.dtype == ZIPVL_BF16) {
@@ -486,7 +505,8 @@ extern "C" zipvl_status zipvl_decode_noalloc(const zipvl_decode_desc *d, const v
         return fail(ZIPVL_ERR_INVALID_ARG, "%s: batch %d heads %d / %d", who, d->batch,
                     d->n_q_heads, d->n_kv_heads);
     if ((d->dtype != ZIPVL_BF16 && d->dtype != ZIPVL_F32 && d->dtype != ZIPVL_F16) ||
-        (d->head_dim != 64 && d->head_dim != 128) || d->n_q_heads / d->n_kv_heads > 8)
+        (d->head_dim != 64 && d->head_dim != 128) ||
+        (d->n_q_heads / d->n_kv_heads > 8 && !decode_tc_supported(*d)))
         return fail(ZIPVL_ERR_UNSUPPORTED, "%s: dtype %d head_dim %d group %d", who, d->dtype,
                     d->head_dim, d->n_q_heads / d->n_kv_heads);
     if (!q || !k_cache || !v_cache || !cache_off || !capacity || !seq_lens || !out)
@@ -529,7 +549,8 @@ extern "C" zipvl_status zipvl_decode_paged(const zipvl_decode_desc *d, const voi
         return fail(ZIPVL_ERR_INVALID_ARG, "%s: batch %d heads %d / %d", who, d->batch,
                     d->n_q_heads, d->n_kv_heads);
     if ((d->dtype != ZIPVL_BF16 && d->dtype != ZIPVL_F32 && d->dtype != ZIPVL_F16) ||
-        (d->head_dim != 64 && d->head_dim != 128) || d->n_q_heads / d->n_kv_heads > 8)
+        (d->head_dim != 64 && d->head_dim != 128) ||
+        (d->n_q_heads / d->n_kv_heads > 8 && !decode_tc_supported(*d)))
         return fail(ZIPVL_ERR_UNSUPPORTED, "%s: dtype %d head_dim %d group %d", who, d->dtype,
                     d->head_dim, d->n_q_heads / d->n_kv_heads);
     if (!q || !k_pages || !v_pages || !block_table || !capacity || !seq_lens || !out || !ws)

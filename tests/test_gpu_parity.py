@@ -716,6 +716,12 @@ def build_caches(lens, Hkv, d, dtype, extra, seed):
     ([90, 257], 4, 4, 64, torch.float16),
     ([300, 7], 4, 4, 64, torch.float32),
     ([129], 6, 2, 128, torch.float32),
+    # grouped-query heads on the tensor cores: 2, 7, 16 and 32 query heads per kv head, an empty
+    # request, lengths of one row, a ragged last tile, more than one chunk per request
+    ([300, 1000], 4, 2, 128, torch.bfloat16),
+    ([5000, 129, 0, 3000, 1], 28, 4, 128, torch.bfloat16),
+    ([2100, 640], 32, 2, 128, torch.float16),
+    ([1500, 127], 32, 1, 128, torch.bfloat16),
 ])
 def test_decode_parity(zipvl, lens, Hq, Hkv, d, dtype):
     B, steps = len(lens), 3
@@ -754,11 +760,45 @@ def test_decode_parity(zipvl, lens, Hq, Hkv, d, dtype):
     assert st.item() & zipvl.DEV_CAPACITY and np.array_equal(seq_d.cpu().numpy(), seq_o)
 
 
+@pytest.mark.parametrize("kernel,lens,Hq,Hkv", [
+    ("tc", [700, 130, 2600], 8, 4),        # two query heads per kv head: the CUDA-core kernel by default
+    ("simt", [700, 130, 2600], 14, 2),     # seven: the tensor-core kernel by default
+    ("tc", [4000], 64, 2),                 # thirty-two, several tiles per CTA
+])
+def test_decode_kernel_choice_can_be_forced_and_both_match_the_oracle(zipvl, monkeypatch, kernel, lens, Hq, Hkv):
+    """ZIPVL_DECODE_KERNEL picks the grouped-query decode kernel; either choice has to match the
+    oracle, repeat bit for bit, and agree with the other one within the attention tolerance."""
+    d, dtype, B = 128, torch.bfloat16, len(lens)
+    kc, vc, off, cap = build_caches(lens, Hkv, d, dtype, 2, seed=7 * sum(lens))
+    g = torch.Generator().manual_seed(5)
+    q = torch.randn(B, Hq, d, generator=g).to(dtype)
+    desc = zipvl.zipvl_decode_desc(B, Hq, Hkv, d, zipvl.ZIPVL_BF16, 0.0)
+    kc_d, vc_d, off_d, cap_d = kc.to(DEV), vc.to(DEV), off.to(DEV), cap.to(DEV)
+    seq_d = torch.tensor(lens, dtype=torch.int32, device=DEV)
+    ref = oracle.decode_step(to_np(q), None, None, kc.float().numpy(), vc.float().numpy(), off.numpy(),
+                             np.array(lens, np.int32), Hkv)
+    outs = {}
+    for which in (kernel, "simt" if kernel == "tc" else "tc"):
+        if Hq // Hkv > 8 and which == "simt":
+            continue                        # more than eight query heads per kv head: tensor cores only
+        monkeypatch.setenv("ZIPVL_DECODE_KERNEL", which)
+        st = status_word()
+        a = zipvl.zipvl_decode(desc, q.to(DEV), None, None, kc_d, vc_d, off_d, cap_d, seq_d, max(lens), status=st)
+        b = zipvl.zipvl_decode(desc, q.to(DEV), None, None, kc_d, vc_d, off_d, cap_d, seq_d, max(lens), status=st)
+        assert st.item() == 0 and torch.equal(a, b)
+        check_attention(to_np(a), ref, dtype)
+        outs[which] = a
+    if len(outs) == 2:
+        check_attention(to_np(outs["tc"]), to_np(outs["simt"]).astype(np.float64), dtype)
+
+
 @pytest.mark.parametrize("lens,Hq,Hkv,d,dtype,page_rows", [
     ([700, 1, 300, 1025, 17, 0], 8, 8, 128, torch.bfloat16, 64),
     ([513, 40, 2000], 14, 2, 128, torch.bfloat16, 128),
     ([100, 259, 64], 4, 1, 64, torch.float16, 16),
     ([300, 7], 4, 4, 64, torch.float32, 64),
+    ([513, 40, 2000, 0], 16, 4, 128, torch.bfloat16, 16),
+    ([3000, 100], 28, 4, 128, torch.float16, 256),
 ])
 def test_paged_decode_parity(zipvl, lens, Hq, Hkv, d, dtype, page_rows):
     """Decode over caches scattered in pages of a shared pool (shuffled page numbers), three
