@@ -71,7 +71,7 @@ typedef struct {
     int32_t L;             /* tokens n */
     int32_t n_q_heads;     /* Hq */
     int32_t n_kv_heads;    /* Hkv, divides Hq */
-    int32_t head_dim;      /* 64 or 128 */
+    int32_t head_dim;      /* 64, 96 or 128: all three run on the tensor cores in 16-bit storage */
     int32_t dtype;         /* ZIPVL_BF16 / ZIPVL_F16 (tensor-core path) or ZIPVL_F32 (true fp32 path) */
     int32_t reserved;
     int64_t q_stride_tok;  /* elements between tokens of Q; 0 = n_q_heads*head_dim */
@@ -214,7 +214,7 @@ zipvl_status zipvl_compact_kv(const zipvl_layer *layer, const void *k, const voi
  * ("O = FlashAttention(Q[T], K[T], V[T])", then "K = K[T], V = V[T]"); both depend only
  * on T.  Results are those of the two calls: out as zipvl_sparse_prefill writes it,
  * k_cache / v_cache / *len_out as zipvl_compact_kv writes them, bit for bit.
- * For bf16, head_dim 128 and a token stride that is a multiple of 16 bytes the copy
+ * For 16-bit storage (head_dim 64, 96 or 128) and a token stride that is a multiple of 16 bytes the copy
  * runs inside the attention kernel (spare warps of each attention CTA copy the key
  * and value rows of that CTA's kept tokens), which takes the compaction off the
  * layer's critical path; other shapes run the two kernels back to back.

@@ -40,8 +40,8 @@ static zipvl_status check_layer(const char *who, const zipvl_layer *l, LayerArgs
         return fail(ZIPVL_ERR_INVALID_ARG, "%s: heads %d / %d", who, l->n_q_heads, l->n_kv_heads);
     if (l->dtype != ZIPVL_BF16 && l->dtype != ZIPVL_F32 && l->dtype != ZIPVL_F16)
         return fail(ZIPVL_ERR_UNSUPPORTED, "%s: dtype %d", who, l->dtype);
-    if (l->head_dim != 64 && l->head_dim != 128)
-        return fail(ZIPVL_ERR_UNSUPPORTED, "%s: head_dim %d (64 or 128)", who, l->head_dim);
+    if (l->head_dim != 64 && l->head_dim != 96 && l->head_dim != 128)
+        return fail(ZIPVL_ERR_UNSUPPORTED, "%s: head_dim %d (64, 96 or 128)", who, l->head_dim);
     const long long qs = l->q_stride_tok ? l->q_stride_tok : (long long)l->n_q_heads * l->head_dim;
     const long long ks = l->kv_stride_tok ? l->kv_stride_tok : (long long)l->n_kv_heads * l->head_dim;
     if (qs < (long long)l->n_q_heads * l->head_dim || ks < (long long)l->n_kv_heads * l->head_dim ||
@@ -233,8 +233,8 @@ zipvl_status zipvl_decode(const zipvl_decode_desc *d, const void *q, const void 
     if (d->batch > 65535) return fail(ZIPVL_ERR_UNSUPPORTED, "zipvl_decode: batch %d > 65535", d->batch);
     if (d->dtype != ZIPVL_BF16 && d->dtype != ZIPVL_F32 && d->dtype != ZIPVL_F16)
         return fail(ZIPVL_ERR_UNSUPPORTED, "zipvl_decode: dtype %d", d->dtype);
-    if (d->head_dim != 64 && d->head_dim != 128)
-        return fail(ZIPVL_ERR_UNSUPPORTED, "zipvl_decode: head_dim %d (64 or 128)", d->head_dim);
+    if (d->head_dim != 64 && d->head_dim != 96 && d->head_dim != 128)
+        return fail(ZIPVL_ERR_UNSUPPORTED, "zipvl_decode: head_dim %d (64, 96 or 128)", d->head_dim);
     if (d->n_q_heads / d->n_kv_heads > 8 && !decode_tc_supported(*d))
         return fail(ZIPVL_ERR_UNSUPPORTED, "zipvl_decode: more than 8 query heads per kv head (up to 32 "
                                            "in 16-bit storage at head_dim 128)");

@@ -67,7 +67,10 @@ decode_kernel(int Hq, int Hkv, float scale_log2, const T *__restrict__ q,
               int chunk, int n_chunks, float *__restrict__ ws, int *__restrict__ lens,
               T *__restrict__ out, int32_t *status_word) {
     constexpr int EPL = Epl<T>::v;          // elements per lane (16 bytes)
-    constexpr int LPR = D / EPL;            // lanes per row
+    constexpr int LPR_USED = D / EPL;       // lanes that hold a piece of a row
+    // lanes per row: a power of two (the dot product is reduced by xor shuffles); with head_dim
+    // 96 the last quarter of them holds nothing
+    constexpr int LPR = LPR_USED <= 8 ? 8 : (LPR_USED <= 16 ? 16 : 32);
     constexpr int RPW = 32 / LPR;           // rows per warp per load
     constexpr int NG = (kDecThreads / 32) * RPW;
     __shared__ float sm_o[NG][GT][D];
@@ -89,7 +92,7 @@ decode_kernel(int Hq, int Hkv, float scale_log2, const T *__restrict__ q,
         const int lr_q = (threadIdx.x & 31) % LPR;
 #pragma unroll
         for (int g = 0; g < GT; ++g) {
-            if (g < n_heads) {
+            if (g < n_heads && lr_q < LPR_USED) {
                 const uint4 r = *reinterpret_cast<const uint4 *>(
                     q + ((long long)b * Hq + h0 + g) * D + lr_q * EPL);
                 unpack<T, EPL>(r, qv[g]);
@@ -122,6 +125,7 @@ decode_kernel(int Hq, int Hkv, float scale_log2, const T *__restrict__ q,
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int rg = warp * RPW + lane / LPR;  // row group of this lane
     const int lr = lane % LPR;               // lane inside the row
+    const bool live = lr < LPR_USED;         // (head_dim 96: 12 of 16 lanes)
 
     if (valid) {
         const int c1 = min(len, c0 + chunk);
@@ -157,7 +161,10 @@ decode_kernel(int Hq, int Hkv, float scale_log2, const T *__restrict__ q,
                 ok[u] = row < c1;
                 const long long ro = ok[u] ? row_off(row) : -1;
                 ok[u] = ok[u] && ro >= 0;
-                if (ok[u] && row != new_row) {
+                if (!live) {
+                    kk[u] = make_uint4(0, 0, 0, 0);
+                    vv[u] = make_uint4(0, 0, 0, 0);
+                } else if (ok[u] && row != new_row) {
                     kk[u] = ld_stream(kb + ro);
                     vv[u] = ld_stream(vb + ro);
                 } else if (ok[u]) {
@@ -221,7 +228,8 @@ decode_kernel(int Hq, int Hkv, float scale_log2, const T *__restrict__ q,
 #pragma unroll
         for (int g = 0; g < GT; ++g) {
 #pragma unroll
-            for (int e = 0; e < EPL; ++e) sm_o[rg][g][lr * EPL + e] = o[g][e];
+            for (int e = 0; e < EPL; ++e)
+                if (live) sm_o[rg][g][lr * EPL + e] = o[g][e];
             if (lr == 0) { sm_m[rg][g] = m[g]; sm_l[rg][g] = l[g]; }
         }
         __syncthreads();
@@ -388,8 +396,10 @@ zipvl_status launch_decode_merge(int dtype, int D, int Hq, int B, int chunk, int
 #define ZIPVL_MERGE(T_, D_) \
     le = launch_dependent(decode_merge_kernel<T_, D_>, grid, dim3(256), 0, st, Hq, chunk, n_chunks, ws, lens, seq_lens, (T_ *)out)
     if (dtype == ZIPVL_BF16 && D == 128) ZIPVL_MERGE(__nv_bfloat16, 128);
+    else if (dtype == ZIPVL_BF16 && D == 96) ZIPVL_MERGE(__nv_bfloat16, 96);
     else if (dtype == ZIPVL_BF16 && D == 64) ZIPVL_MERGE(__nv_bfloat16, 64);
     else if (dtype == ZIPVL_F16 && D == 128) ZIPVL_MERGE(__half, 128);
+    else if (dtype == ZIPVL_F16 && D == 96) ZIPVL_MERGE(__half, 96);
     else if (dtype == ZIPVL_F16 && D == 64) ZIPVL_MERGE(__half, 64);
 #undef ZIPVL_MERGE
     if (le != cudaSuccess) return fail(ZIPVL_ERR_CUDA, "decode merge: launch: %s", cudaGetErrorString(le));
@@ -435,12 +445,15 @@ zipvl_status dispatch_decode(const zipvl_decode_desc &d, float scale_log2, const
                    seq_lens, max_len, out, ws, status_word, st
     if (d.dtype == ZIPVL_BF16) {
         if (d.head_dim == 128) return run<__nv_bfloat16, 128>(ZIPVL_ARGS);
+        if (d.head_dim == 96) return run<__nv_bfloat16, 96>(ZIPVL_ARGS);
         if (d.head_dim == 64) return run<__nv_bfloat16, 64>(ZIPVL_ARGS);
     } else if (d.dtype == ZIPVL_F16) {
         if (d.head_dim == 128) return run<__half, 128>(ZIPVL_ARGS);
+        if (d.head_dim == 96) return run<__half, 96>(ZIPVL_ARGS);
         if (d.head_dim == 64) return run<__half, 64>(ZIPVL_ARGS);
     } else {
         if (d.head_dim == 128) return run<float, 128>(ZIPVL_ARGS);
+        if (d.head_dim == 96) return run<float, 96>(ZIPVL_ARGS);
         if (d.head_dim == 64) return run<float, 64>(ZIPVL_ARGS);
     }
 #undef ZIPVL_ARGS
@@ -505,7 +518,7 @@ extern "C" zipvl_status zipvl_decode_noalloc(const zipvl_decode_desc *d, const v
         return fail(ZIPVL_ERR_INVALID_ARG, "%s: batch %d heads %d / %d", who, d->batch,
                     d->n_q_heads, d->n_kv_heads);
     if ((d->dtype != ZIPVL_BF16 && d->dtype != ZIPVL_F32 && d->dtype != ZIPVL_F16) ||
-        (d->head_dim != 64 && d->head_dim != 128) ||
+        (d->head_dim != 64 && d->head_dim != 96 && d->head_dim != 128) ||
         (d->n_q_heads / d->n_kv_heads > 8 && !decode_tc_supported(*d)))
         return fail(ZIPVL_ERR_UNSUPPORTED, "%s: dtype %d head_dim %d group %d", who, d->dtype,
                     d->head_dim, d->n_q_heads / d->n_kv_heads);
@@ -549,7 +562,7 @@ extern "C" zipvl_status zipvl_decode_paged(const zipvl_decode_desc *d, const voi
         return fail(ZIPVL_ERR_INVALID_ARG, "%s: batch %d heads %d / %d", who, d->batch,
                     d->n_q_heads, d->n_kv_heads);
     if ((d->dtype != ZIPVL_BF16 && d->dtype != ZIPVL_F32 && d->dtype != ZIPVL_F16) ||
-        (d->head_dim != 64 && d->head_dim != 128) ||
+        (d->head_dim != 64 && d->head_dim != 96 && d->head_dim != 128) ||
         (d->n_q_heads / d->n_kv_heads > 8 && !decode_tc_supported(*d)))
         return fail(ZIPVL_ERR_UNSUPPORTED, "%s: dtype %d head_dim %d group %d", who, d->dtype,
                     d->head_dim, d->n_q_heads / d->n_kv_heads);

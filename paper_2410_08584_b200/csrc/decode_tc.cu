@@ -49,7 +49,10 @@ constexpr int kGroups = ZIPVL_DT_GROUPS;
 // (every use of a ring slot must fall to the same group, which fills its tiles in order: a
 // slot's "empty" barrier is then never more than one phase behind its reader)
 static_assert(6 % ZIPVL_DT_GROUPS == 0, "a group owns whole ring slots");
-constexpr int kWindow = 3;             // tile loads in flight per producer thread
+#ifndef ZIPVL_DT_WINDOW
+#define ZIPVL_DT_WINDOW 3
+#endif
+constexpr int kWindow = ZIPVL_DT_WINDOW;             // tile loads in flight per producer thread
 constexpr int kIssuerWarp = 4 + 4 * kGroups;
 constexpr int kHalfBytes = 128 * 128;
 constexpr int kTileBytes = 2 * kHalfBytes;

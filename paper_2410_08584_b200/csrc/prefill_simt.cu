@@ -209,12 +209,15 @@ zipvl_status launch_prefill_simt(const LayerArgs &a, int dtype, const void *q, c
                                  cudaStream_t st) {
     if (dtype == ZIPVL_F32) {
         if (a.D == 64) return run<float, 64>(a, q, k, v, idx, k_dev, k_max, out, out_mode, status_word, st);
+        if (a.D == 96) return run<float, 96>(a, q, k, v, idx, k_dev, k_max, out, out_mode, status_word, st);
         if (a.D == 128) return run<float, 128>(a, q, k, v, idx, k_dev, k_max, out, out_mode, status_word, st);
     } else if (dtype == ZIPVL_F16) {
         if (a.D == 64) return run<__half, 64>(a, q, k, v, idx, k_dev, k_max, out, out_mode, status_word, st);
+        if (a.D == 96) return run<__half, 96>(a, q, k, v, idx, k_dev, k_max, out, out_mode, status_word, st);
         if (a.D == 128) return run<__half, 128>(a, q, k, v, idx, k_dev, k_max, out, out_mode, status_word, st);
     } else {
         if (a.D == 64) return run<__nv_bfloat16, 64>(a, q, k, v, idx, k_dev, k_max, out, out_mode, status_word, st);
+        if (a.D == 96) return run<__nv_bfloat16, 96>(a, q, k, v, idx, k_dev, k_max, out, out_mode, status_word, st);
         if (a.D == 128) return run<__nv_bfloat16, 128>(a, q, k, v, idx, k_dev, k_max, out, out_mode, status_word, st);
     }
     return fail(ZIPVL_ERR_UNSUPPORTED, "sparse_prefill: head_dim %d", a.D);

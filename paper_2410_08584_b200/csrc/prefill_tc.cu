@@ -42,7 +42,7 @@ namespace {
 
 using namespace ptx;
 
-constexpr int kD = 128;               // head_dim
+constexpr int kD = 128;               // width of the shared-memory tiles; head_dim 64 and 96 use the front of it
 constexpr int kBM = 128, kBN = 128;   // query / key tile
 constexpr int kPair = 2 * kBM;        // query rows per CTA
 constexpr int kSlots = 5;             // ring of K / V tiles
@@ -80,12 +80,15 @@ constexpr size_t kSmemBytes = kTileBytes * (2 + kSlots) + sizeof(Barriers) + 102
 // 32-byte sectors of two rows.  The loop is the producers' whole instruction stream
 // and they share their schedulers with the softmax warps, so it is kept to a
 // shuffle, one multiply-add for the source, one xor for the swizzle and the copy.
-template <bool kAllValid>
+template <bool kAllValid, int n_chunks16>
 __device__ __forceinline__ void gather_rows32_impl(uint32_t tile, int row0, int my_tok,
                                                    const __nv_bfloat16 *base, unsigned int stride_bytes,
                                                    int lane) {
     const int c = lane & 15, sub = lane >> 4;
-    const char *src_lane = reinterpret_cast<const char *>(base) + c * 16;
+    // a row of head_dim 64 or 96 has 8 or 12 chunks: the other lanes copy nothing (zero-fill of
+    // columns no MMA reads) and never look past the row
+    const uint32_t lane_bytes = (n_chunks16 == 16 || c < n_chunks16) ? 16u : 0u;
+    const char *src_lane = reinterpret_cast<const char *>(base) + ((n_chunks16 == 16 || c < n_chunks16) ? c : 0) * 16;
     // every term but the chunk is a multiple of 128: the swizzle is an xor of the low bits
     const uint32_t dst_lane = (tile + (row0 + 16 * sub) * 128 + (c >> 3) * kHalfBytes) | ((c & 7) << 4);
 #pragma unroll
@@ -93,23 +96,28 @@ __device__ __forceinline__ void gather_rows32_impl(uint32_t tile, int row0, int 
         const int t = __shfl_sync(0xffffffffu, my_tok, i, 16);        // row i of my half-warp
         const uint32_t dst = (dst_lane ^ ((i & 7) << 4)) + i * 128;
         if (kAllValid)
-            cp_async16(dst, src_lane + (unsigned long long)(unsigned int)t * stride_bytes, 16u);
+            cp_async16(dst, src_lane + (unsigned long long)(unsigned int)t * stride_bytes, lane_bytes);
         else
             cp_async16(dst, src_lane + (unsigned long long)(unsigned int)(t < 0 ? 0 : t) * stride_bytes,
-                       t >= 0 ? 16u : 0u);
+                       t >= 0 ? lane_bytes : 0u);
     }
 }
+template <int n_chunks16>
 __device__ __forceinline__ void gather_rows32(uint32_t tile, int row0, int my_tok,
                                               const __nv_bfloat16 *base, long long stride,
                                               int lane) {
     const unsigned int stride_bytes = (unsigned int)(stride * 2);     // (checked by the host: < 2^31)
-    if (__all_sync(0xffffffffu, my_tok >= 0)) gather_rows32_impl<true>(tile, row0, my_tok, base, stride_bytes, lane);
-    else gather_rows32_impl<false>(tile, row0, my_tok, base, stride_bytes, lane);
+    if (__all_sync(0xffffffffu, my_tok >= 0))
+        gather_rows32_impl<true, n_chunks16>(tile, row0, my_tok, base, stride_bytes, lane);
+    else
+        gather_rows32_impl<false, n_chunks16>(tile, row0, my_tok, base, stride_bytes, lane);
 }
 
 // kHalf: the 16-bit storage type is IEEE half instead of bfloat16 (pointers are typed
 // __nv_bfloat16 either way: only their width matters to the loads and stores)
-template <bool kHalf>
+// kHd: head_dim (64, 96 or 128), a compile-time constant so that the 128 instantiation carries
+// none of the narrower rows' tests
+template <bool kHalf, int kHd>
 __global__ void __launch_bounds__(kThreadsTc, 1)
 prefill_tc_kernel(LayerArgs a, const __nv_bfloat16 *__restrict__ q,
                   const __nv_bfloat16 *__restrict__ k, const __nv_bfloat16 *__restrict__ v,
@@ -150,15 +158,16 @@ prefill_tc_kernel(LayerArgs a, const __nv_bfloat16 *__restrict__ q,
     // grid.x = query head + Hq * sequence: every sequence of a batch has its own tensors, index
     // list, k, output and cache, stacked; its heaviest pairs still start first
     const int h = blockIdx.x % a.Hq, g = h / a.G;
+    constexpr int nch = kHd >> 3;            // 16-byte chunks of a row
     {
         const int z = blockIdx.x / a.Hq;
         q += z * a.q_seq; k += z * a.kv_seq; v += z * a.kv_seq;
         idx += (long long)z * a.L;
         k_dev += z;
-        out += (long long)z * (out_mode == ZIPVL_OUT_PADDED ? a.L : k_max) * a.Hq * kD;
+        out += (long long)z * (out_mode == ZIPVL_OUT_PADDED ? a.L : k_max) * a.Hq * kHd;
         if (kc != nullptr) {
-            kc += (long long)z * capacity * a.Hkv * kD;
-            vc += (long long)z * capacity * a.Hkv * kD;
+            kc += (long long)z * capacity * a.Hkv * kHd;
+            vc += (long long)z * capacity * a.Hkv * kHd;
             len_out += z;
         }
     }
@@ -213,7 +222,8 @@ prefill_tc_kernel(LayerArgs a, const __nv_bfloat16 *__restrict__ q,
             if (out_mode == ZIPVL_OUT_PADDED) {
                 const uint4 z = make_uint4(0, 0, 0, 0);
                 for (int e = threadIdx.x; e < a.L * 16; e += kThreadsTc)
-                    reinterpret_cast<uint4 *>(out + ((long long)(e >> 4) * a.Hq + h) * kD)[e & 15] = z;
+                    if ((e & 15) < nch)
+                        reinterpret_cast<uint4 *>(out + ((long long)(e >> 4) * a.Hq + h) * kHd)[e & 15] = z;
             }
             if (kc != nullptr && h == 0 && threadIdx.x == 0) *len_out = 0;
         }
@@ -229,8 +239,8 @@ prefill_tc_kernel(LayerArgs a, const __nv_bfloat16 *__restrict__ q,
         auto issue = [&](int seq) {
             const int slot = seq % kSlots;
             if ((seq & 1) == 0 && seq > 0) tok = token_of((seq >> 1) * kBN + row0 + lane);
-            const __nv_bfloat16 *src = ((seq & 1) ? v : k) + (long long)g * kD;
-            gather_rows32(sRing + slot * kTileBytes, row0, tok, src, a.kv_stride, lane);
+            const __nv_bfloat16 *src = ((seq & 1) ? v : k) + (long long)g * kHd;
+            gather_rows32<nch>(sRing + slot * kTileBytes, row0, tok, src, a.kv_stride, lane);
             cp_async_commit();
         };
         auto slot_free = [&](int seq, bool block) {
@@ -268,8 +278,9 @@ prefill_tc_kernel(LayerArgs a, const __nv_bfloat16 *__restrict__ q,
                 const uint4 z = make_uint4(0, 0, 0, 0);
                 const int sub = lane >> 4, ch = lane & 15;
                 auto clear_rows = [&](int r0, int r1) {
-                    for (int zr = r0 + sub; zr < r1; zr += 2)
-                        reinterpret_cast<uint4 *>(out + ((long long)zr * a.Hq + h) * kD)[ch] = z;
+                    if (ch < nch)
+                        for (int zr = r0 + sub; zr < r1; zr += 2)
+                            reinterpret_cast<uint4 *>(out + ((long long)zr * a.Hq + h) * kHd)[ch] = z;
                 };
                 for (int i0 = (warp - 13) * 32; i0 < (has_b ? kPair : kBM); i0 += 3 * 32) {
                     const int i = q0 + i0 + lane;
@@ -318,10 +329,10 @@ prefill_tc_kernel(LayerArgs a, const __nv_bfloat16 *__restrict__ q,
                         __nv_bfloat16 *dstc = kind ? vc : kc;
                         for (int r = (warp - 13) * 2 + sub; r < kBN; r += 3 * 2) {
                             const int i = j * kBN + r;
-                            if (i >= lim) continue;    // (a row with an invalid index is all zeros here)
+                            if (i >= lim || ch >= nch) continue;    // (a row with an invalid index is all zeros here)
                             const uint4 w = *reinterpret_cast<const uint4 *>(
                                 tile + (ch >> 3) * kHalfBytes + r * 128 + (((ch & 7) ^ (r & 7)) << 4));
-                            reinterpret_cast<uint4 *>(dstc + ((long long)i * a.Hkv + g) * kD)[ch] = w;
+                            reinterpret_cast<uint4 *>(dstc + ((long long)i * a.Hkv + g) * kHd)[ch] = w;
                         }
                     }
                 }
@@ -336,7 +347,7 @@ prefill_tc_kernel(LayerArgs a, const __nv_bfloat16 *__restrict__ q,
             // and stays in uniform registers); one elected lane issues.
             const bool leader = elect_one();
             constexpr uint32_t idesc_qk = idesc_f16kind(kBM, kBN, false, false, !kHalf);
-            constexpr uint32_t idesc_pv = idesc_f16kind(kBM, kD, false, true, !kHalf);
+            constexpr uint32_t idesc_pv = idesc_f16kind(kBM, kHd, false, true, !kHalf);   // N = head_dim
             // Descriptors are built once: the high word is constant (SBO 1024 B,
             // version, 128-byte swizzle); the low word is (address >> 4) | LBO << 16
             // and moves by a compile-time offset per k-block, so issuing one MMA is
@@ -357,7 +368,7 @@ prefill_tc_kernel(LayerArgs a, const __nv_bfloat16 *__restrict__ q,
                 const uint32_t d = tmem + x * 128;
                 if (leader) {
 #pragma unroll
-                    for (int kb = 0; kb < kD / 16; ++kb) {
+                    for (int kb = 0; kb < kHd / 16; ++kb) {
                         const uint32_t o = ((kb >> 2) * kHalfBytes + (kb & 3) * 32) >> 4;
                         mma_ss(d, desc(lo_q + o), desc(lo_k + o), idesc_qk, kb > 0);
                     }
@@ -436,8 +447,8 @@ prefill_tc_kernel(LayerArgs a, const __nv_bfloat16 *__restrict__ q,
         const int x = warp >> 2;                        // 0 = tile A, 1 = tile B
         const int row = threadIdx.x & 127;              // TMEM lane, query row in tile
         // every warp gathers its own 32 query rows (rows past the kept set are zero-filled)
-        gather_rows32(sQ + x * kTileBytes, (warp & 3) * 32, first_tok, q + (long long)h * kD, a.q_stride,
-                      lane);
+        gather_rows32<nch>(sQ + x * kTileBytes, (warp & 3) * 32, first_tok, q + (long long)h * kHd, a.q_stride,
+                           lane);
         cp_async_commit();
         cp_async_wait<0>();
         fence_proxy_async();
@@ -532,7 +543,7 @@ prefill_tc_kernel(LayerArgs a, const __nv_bfloat16 *__restrict__ q,
                     // O is complete through tile n-1: the commit that announced S(n) was
                     // issued after PV(n-1) and covers it
 #pragma unroll 1
-                    for (int c = 0; c < 4; ++c) {
+                    for (int c = 0; c < (kHd >> 5); ++c) {
                         uint32_t r[32];
                         tmem_ld32(tO + c * 32, r);
                         tmem_wait_ld();
@@ -561,7 +572,7 @@ prefill_tc_kernel(LayerArgs a, const __nv_bfloat16 *__restrict__ q,
             const bool padded = (out_mode == ZIPVL_OUT_PADDED);
             __nv_bfloat16 *dst = nullptr;
             if (t >= 0 && !*abort_flag)
-                dst = out + ((long long)(padded ? t : i) * a.Hq + h) * kD;
+                dst = out + ((long long)(padded ? t : i) * a.Hq + h) * kHd;
             // The normalised row goes to global memory through this tile's query buffer
             // (no MMA reads it any more: the last score tile has landed).  Each warp stages
             // its own 32 rows -- a lane writes its row, 16-byte chunks XOR-swizzled by the row
@@ -569,7 +580,7 @@ prefill_tc_kernel(LayerArgs a, const __nv_bfloat16 *__restrict__ q,
             // per instruction, 16 lanes covering one contiguous 256-byte row.
             unsigned char *stage = gen + (size_t)x * kTileBytes + (size_t)(warp & 3) * (32 * 256);
 #pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
+            for (int c = 0; c < (kHd >> 5); ++c) {
                 uint32_t r[32];
                 tmem_ld32(tO + c * 32, r);
                 tmem_wait_ld();
@@ -592,7 +603,7 @@ prefill_tc_kernel(LayerArgs a, const __nv_bfloat16 *__restrict__ q,
                     // destination of row rr of this warp: its lane holds the pointer
                     const unsigned long long d = __shfl_sync(0xffffffffu, (unsigned long long)dst, rr);
                     const uint4 w = *reinterpret_cast<const uint4 *>(stage + rr * 256 + ((ch ^ (rr & 15)) << 4));
-                    if (d) reinterpret_cast<uint4 *>(d)[ch] = w;
+                    if (d && ch < nch) reinterpret_cast<uint4 *>(d)[ch] = w;
                 }
             }
         }
@@ -611,7 +622,8 @@ prefill_tc_kernel(LayerArgs a, const __nv_bfloat16 *__restrict__ q,
 
 bool prefill_tc_supported(const LayerArgs &a, int dtype) {
     // (row strides in bytes are kept in 32 bits by the gathers)
-    return (dtype == ZIPVL_BF16 || dtype == ZIPVL_F16) && a.D == 128 && a.q_stride < (1ll << 30) &&
+    return (dtype == ZIPVL_BF16 || dtype == ZIPVL_F16) && (a.D == 128 || a.D == 96 || a.D == 64) &&
+           a.q_stride < (1ll << 30) &&
            a.kv_stride < (1ll << 30);
 }
 
@@ -632,10 +644,12 @@ zipvl_status launch_prefill_tc(const LayerArgs &a, const void *q, const void *k,
     const char *env = getenv("ZIPVL_PREFILL_KERNEL");
     const int forced = !env ? 0 : (!strcmp(env, "pair") ? 1 : (!strcmp(env, "single") ? 2 : 0));
     const bool single = forced ? (forced == 2) : ((long long)k_max * a.Hq <= kSingleTileMaxRows);
-    if (single && a.n_seq == 1)
+    if (single && a.n_seq == 1 && a.D == 128)
         return launch_prefill_tc1(a, q, k, v, idx, k_dev, k_max, out, out_mode, k_cache, v_cache,
                                   capacity, len_out, status_word, st);
-    auto kernel = a.half ? prefill_tc_kernel<true> : prefill_tc_kernel<false>;
+    auto kernel = a.half ? prefill_tc_kernel<true, 128> : prefill_tc_kernel<false, 128>;
+    if (a.D == 96) kernel = a.half ? prefill_tc_kernel<true, 96> : prefill_tc_kernel<false, 96>;
+    if (a.D == 64) kernel = a.half ? prefill_tc_kernel<true, 64> : prefill_tc_kernel<false, 64>;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
     if (e != cudaSuccess)
         return fail(ZIPVL_ERR_CUDA, "sparse_prefill: smem opt-in: %s", cudaGetErrorString(e));

@@ -262,12 +262,15 @@ zipvl_status launch_score_simt(const LayerArgs &a, int dtype, const void *q, con
     if (P > 8192) return fail(ZIPVL_ERR_UNSUPPORTED, "score: n_probe %d > 8192", P);
     if (dtype == ZIPVL_F32) {
         if (a.D == 64) return run<float, 64>(a, q, k, probe_pos, P, acc, norm, total, ws, status_word, st);
+        if (a.D == 96) return run<float, 96>(a, q, k, probe_pos, P, acc, norm, total, ws, status_word, st);
         if (a.D == 128) return run<float, 128>(a, q, k, probe_pos, P, acc, norm, total, ws, status_word, st);
     } else if (dtype == ZIPVL_F16) {
         if (a.D == 64) return run<__half, 64>(a, q, k, probe_pos, P, acc, norm, total, ws, status_word, st);
+        if (a.D == 96) return run<__half, 96>(a, q, k, probe_pos, P, acc, norm, total, ws, status_word, st);
         if (a.D == 128) return run<__half, 128>(a, q, k, probe_pos, P, acc, norm, total, ws, status_word, st);
     } else {
         if (a.D == 64) return run<__nv_bfloat16, 64>(a, q, k, probe_pos, P, acc, norm, total, ws, status_word, st);
+        if (a.D == 96) return run<__nv_bfloat16, 96>(a, q, k, probe_pos, P, acc, norm, total, ws, status_word, st);
         if (a.D == 128) return run<__nv_bfloat16, 128>(a, q, k, probe_pos, P, acc, norm, total, ws, status_word, st);
     }
     return fail(ZIPVL_ERR_UNSUPPORTED, "score: head_dim %d", a.D);

@@ -1,6 +1,6 @@
 // Probe scoring on the tensor cores (supplementary Eq. A with the causal mask of
-// Eq. 2; column sums of Eq. 6; normalisation of Eq. 8).  bf16 or fp16, head_dim 128,
-// up to 128 probe rows.
+// Eq. 2; column sums of Eq. 6; normalisation of Eq. 8).  bf16 or fp16, head_dim 64, 96 or
+// 128, up to 128 probe rows.
 //
 // A column sum of a row-softmax needs each row's final max and denominator, so
 // the probe x key contraction runs twice; the attention matrix only ever exists
@@ -27,6 +27,8 @@ namespace {
 
 using namespace ptx;
 
+// kD: the width of the shared-memory tiles (two 64-column swizzle atoms); head_dim 64 and 96 use
+// the front of it -- fewer 16-byte chunks per gathered row, fewer k-blocks per MMA
 constexpr int kD = 128, kTile = 128, kMaxProbe = 128;
 constexpr int kHalfBytes = 128 * 128;
 constexpr int kTileBytes = 2 * kHalfBytes;
@@ -46,6 +48,7 @@ struct ScBarriers {
 
 constexpr size_t kScSmem = kTileBytes * (1 + kKStages) + 3 * kMaxProbe * 4 + sizeof(ScBarriers) + 1024;
 
+template <int n_chunks16>
 __device__ __forceinline__ void gather_row_sw128(uint32_t tile, int row, const __nv_bfloat16 *src,
                                                  bool valid) {
     const uint32_t bytes = valid ? 16u : 0u;
@@ -53,14 +56,16 @@ __device__ __forceinline__ void gather_row_sw128(uint32_t tile, int row, const _
     const int sw = row & 7;
 #pragma unroll
     for (int c = 0; c < 16; ++c)
-        cp_async16(rbase + (c >> 3) * kHalfBytes + (((c & 7) ^ sw) << 4), src + c * 8, bytes);
+        if (c < n_chunks16)
+            cp_async16(rbase + (c >> 3) * kHalfBytes + (((c & 7) ^ sw) << 4), src + c * 8, bytes);
 }
 
 // MODE 0: row statistics.  MODE 1: column sums.
 // barrier over the 128 consumer threads only (named barrier 1)
 __device__ __forceinline__ void consumer_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
-template <int MODE>
+// kHd: head_dim (64, 96 or 128) as a compile-time constant
+template <int MODE, int kHd>
 __global__ void __launch_bounds__(kThreadsSc, 2)   // two CTAs per SM hide each other's latency
 score_tc_kernel(const __grid_constant__ CUtensorMap kmap, LayerArgs a,
                 const __nv_bfloat16 *__restrict__ q, const int32_t *__restrict__ probe_pos, int P,
@@ -125,7 +130,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap kmap, LayerArgs a,
         sPos[r] = c;
         // this thread's probe row is requested at once (it lands while the barriers and
         // the tensor memory are set up); the row is announced after the barrier below
-        gather_row_sw128(sQ, r, q + (long long)(c < 0 ? 0 : c) * a.q_stride + (long long)h * kD, c >= 0);
+        gather_row_sw128<(kHd >> 3)>(sQ, r, q + (long long)(c < 0 ? 0 : c) * a.q_stride + (long long)h * kHd, c >= 0);
         cp_async_commit();
     }
     tc_fence_before();
@@ -143,11 +148,13 @@ score_tc_kernel(const __grid_constant__ CUtensorMap kmap, LayerArgs a,
                     mbar_wait(smem_u32(&bar->k_empty[s]), ((n / kKStages) - 1) & 1, abort_flag);
                 if (*abort_flag) break;
                 const uint32_t fb = smem_u32(&bar->k_full[s]);
-                mbar_expect_tx(fb, kTileBytes);
+                // (head_dim 96: the second box runs 32 columns into the next head, or past the
+                // row, where the copy fills zeros; no MMA reads those columns)
+                mbar_expect_tx(fb, kHd > 64 ? kTileBytes : kHalfBytes);
                 const uint32_t dst = sK + s * kTileBytes;
                 const int y = z * a.L + (t0 + n) * kTile;
-                tma_load_2d(dst, &kmap, g * kD, y, fb);
-                tma_load_2d(dst + kHalfBytes, &kmap, g * kD + 64, y, fb);
+                tma_load_2d(dst, &kmap, g * kHd, y, fb);
+                if (kHd > 64) tma_load_2d(dst + kHalfBytes, &kmap, g * kHd + 64, y, fb);
             }
         }
     } else if (warp == 5) {
@@ -170,7 +177,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap kmap, LayerArgs a,
             if (leader) {
                 if (!*abort_flag) {
 #pragma unroll
-                    for (int kb = 0; kb < kD / 16; ++kb) {
+                    for (int kb = 0; kb < kHd / 16; ++kb) {
                         const uint32_t o = ((kb >> 2) * kHalfBytes + (kb & 3) * 32) >> 4;
                         const uint64_t dq = ((uint64_t)kDescHi << 32) | (lo_q + o);
                         const uint64_t dk = ((uint64_t)kDescHi << 32) | (lo_k + o);
@@ -395,7 +402,8 @@ int tiles_per_chunk_for(int L, int Hq) {
 __global__ void sum_to_double_kernel(int L, const float *__restrict__ x, double *__restrict__ out);
 
 bool score_tc_supported(const LayerArgs &a, int dtype, int n_probe) {
-    return (dtype == ZIPVL_BF16 || dtype == ZIPVL_F16) && a.D == 128 && n_probe <= kMaxProbe &&
+    return (dtype == ZIPVL_BF16 || dtype == ZIPVL_F16) && (a.D == 128 || a.D == 96 || a.D == 64) &&
+           n_probe <= kMaxProbe &&
            encode_tiled_fn() != nullptr;
 }
 
@@ -437,20 +445,27 @@ zipvl_status launch_score_tc(const LayerArgs &a, const void *q, const void *k,
                                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (cr != CUDA_SUCCESS) return fail(ZIPVL_ERR_CUDA, "score: cuTensorMapEncodeTiled failed (%d)", (int)cr);
 
-    cudaError_t e = cudaFuncSetAttribute(score_tc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kScSmem);
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(score_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kScSmem);
-    if (e != cudaSuccess) return fail(ZIPVL_ERR_CUDA, "score: smem opt-in: %s", cudaGetErrorString(e));
-
     const __nv_bfloat16 *qb = (const __nv_bfloat16 *)q;
     dim3 grid(n_chunks, a.Hq, a.n_seq);
+    cudaError_t e = cudaSuccess;
     // both launches are programmatic dependents: <1> may begin its set-up, loads and first
     // MMA while <0> drains, and <0> itself may be staged behind the caller's previous kernel
-    e = launch_dependent(score_tc_kernel<0>, grid, dim3(kThreadsSc), kScSmem, st, kmap, a, qb, probe_pos, P,
-                         tpc, n_chunks, stats, partial, counters, acc, norm, status_word);
-    if (e == cudaSuccess)
-        e = launch_dependent(score_tc_kernel<1>, grid, dim3(kThreadsSc), kScSmem, st, kmap, a, qb, probe_pos,
-                             P, tpc, n_chunks, stats, partial, counters, acc, norm, status_word);
+#define ZIPVL_SCORE_LAUNCH(HD_)                                                                      \
+    {                                                                                                \
+        e = cudaFuncSetAttribute(score_tc_kernel<0, HD_>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kScSmem); \
+        if (e == cudaSuccess)                                                                        \
+            e = cudaFuncSetAttribute(score_tc_kernel<1, HD_>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kScSmem); \
+        if (e != cudaSuccess) return fail(ZIPVL_ERR_CUDA, "score: smem opt-in: %s", cudaGetErrorString(e)); \
+        e = launch_dependent(score_tc_kernel<0, HD_>, grid, dim3(kThreadsSc), kScSmem, st, kmap, a, qb, probe_pos, P, \
+                             tpc, n_chunks, stats, partial, counters, acc, norm, status_word);       \
+        if (e == cudaSuccess)                                                                        \
+            e = launch_dependent(score_tc_kernel<1, HD_>, grid, dim3(kThreadsSc), kScSmem, st, kmap, a, qb, probe_pos, \
+                                 P, tpc, n_chunks, stats, partial, counters, acc, norm, status_word); \
+    }
+    if (a.D == 128) ZIPVL_SCORE_LAUNCH(128)
+    else if (a.D == 96) ZIPVL_SCORE_LAUNCH(96)
+    else ZIPVL_SCORE_LAUNCH(64)
+#undef ZIPVL_SCORE_LAUNCH
     if (e != cudaSuccess) return fail(ZIPVL_ERR_CUDA, "score: launch: %s", cudaGetErrorString(e));
     if (total)
         for (int z = 0; z < a.n_seq; ++z) sum_to_double_kernel<<<1, 1024, 0, st>>>(a.L, acc + (size_t)z * a.L, total + z);

@@ -28,6 +28,12 @@ def layer_cases():
         "llava7b_small_fp16": lambda: W.heavy_key_layer(L_visual=1150, L_text=64, H=8, seed=31,
                                                         dtype=torch.float16),
         "fp16_d64": lambda: W.heavy_key_layer(L_visual=300, L_text=33, H=4, d=64, seed=32, dtype=torch.float16),
+        # head_dim 96 and 64 on the tensor-core kernels (the front of their 128-wide tiles), with
+        # grouped heads and several key tiles; head_dim 96 in fp32 on the CUDA-core kernels
+        "bf16_d96_gqa": lambda: W.heavy_key_layer(L_visual=1200, L_text=77, H=6, Hkv=2, d=96, seed=41),
+        "fp16_d96": lambda: W.heavy_key_layer(L_visual=400, L_text=19, H=3, d=96, seed=42, dtype=torch.float16),
+        "bf16_d64_gqa": lambda: W.heavy_key_layer(L_visual=1300, L_text=64, H=8, Hkv=4, d=64, seed=43),
+        "fp32_d96": lambda: W.tiny_layer(L=300, H=2, d=96, n_probe=40, seed=44),
         "video_gqa_small_fp16": lambda: W.video_layer(n_frames=7, Hq=14, Hkv=2, seed=33, dtype=torch.float16),
     }
 
@@ -716,6 +722,9 @@ def build_caches(lens, Hkv, d, dtype, extra, seed):
     ([90, 257], 4, 4, 64, torch.float16),
     ([300, 7], 4, 4, 64, torch.float32),
     ([129], 6, 2, 128, torch.float32),
+    ([400, 130, 1], 6, 2, 96, torch.bfloat16),
+    ([257, 90], 4, 4, 96, torch.float16),
+    ([300, 7], 4, 2, 96, torch.float32),
     # grouped-query heads on the tensor cores: 2, 7, 16 and 32 query heads per kv head, an empty
     # request, lengths of one row, a ragged last tile, more than one chunk per request
     ([300, 1000], 4, 2, 128, torch.bfloat16),
@@ -797,6 +806,7 @@ def test_decode_kernel_choice_can_be_forced_and_both_match_the_oracle(zipvl, mon
     ([513, 40, 2000], 14, 2, 128, torch.bfloat16, 128),
     ([100, 259, 64], 4, 1, 64, torch.float16, 16),
     ([300, 7], 4, 4, 64, torch.float32, 64),
+    ([300, 70], 6, 2, 96, torch.bfloat16, 32),
     ([513, 40, 2000, 0], 16, 4, 128, torch.bfloat16, 16),
     ([3000, 100], 28, 4, 128, torch.float16, 256),
 ])
