@@ -650,6 +650,72 @@ def decode_benchmark(z, dev, steps, peaks, B=16, ctx_max=32768):
     return res
 
 
+def decode_gqa_benchmark(z, dev, peaks, steps=64, B=16, Hq=28, Hkv=4, d=128):
+    """Grouped-query decode (the long-video model's head shape: 28 query heads on 4 kv heads) on kept
+    caches of 6K-30K rows: the tensor-core kernel (default from three query heads per kv head) next to
+    the CUDA-core kernel, which ZIPVL_DECODE_KERNEL selects; one request checked against the oracle."""
+    import oracle
+    g = torch.Generator().manual_seed(BASE_SEED + 6)
+    lens = torch.randint(6000, 30001, (B,), generator=g).tolist()
+    row = Hkv * d
+    caps = [n + steps + 1 for n in lens]
+    gd = torch.Generator(device=dev).manual_seed(BASE_SEED + 6)
+    kcache = torch.randn(sum(caps) * row, generator=gd, device=dev).bfloat16()
+    vcache = torch.randn(sum(caps) * row, generator=gd, device=dev).bfloat16()
+    off = torch.tensor(np.concatenate([[0], np.cumsum([c * row for c in caps[:-1]])]), dtype=torch.int64, device=dev)
+    capt = torch.tensor(caps, dtype=torch.int32, device=dev)
+    max_len = max(caps)
+    ddesc = z.zipvl_decode_desc(B, Hq, Hkv, d, z.ZIPVL_BF16, 0.0)
+    dl = z.zipvl_layer(max_len, Hq, Hkv, d, z.ZIPVL_BF16, 0, 0, 0, 0.0, 0)
+    ws = z.workspace(z.zipvl_workspace_bytes(z.OP_DECODE, dl, 0, B), dev)
+    n_rot = 4
+    qs = torch.randn(n_rot, B, Hq, d, generator=gd, device=dev).bfloat16()
+    kn = torch.randn(n_rot, B, Hkv, d, generator=gd, device=dev).bfloat16()
+    vn = torch.randn(n_rot, B, Hkv, d, generator=gd, device=dev).bfloat16()
+    out = torch.empty(B, Hq, d, dtype=torch.bfloat16, device=dev)
+    res = {"batch": B, "n_q_heads": Hq, "n_kv_heads": Hkv, "lens": lens, "steps": steps}
+    prev = os.environ.get("ZIPVL_DECODE_KERNEL")
+    try:
+        for name in ("tensor_core", "cuda_core"):
+            os.environ["ZIPVL_DECODE_KERNEL"] = "tc" if name == "tensor_core" else "simt"
+            seq = torch.tensor(lens, dtype=torch.int32, device=dev)
+            st = torch.zeros(1, dtype=torch.int32, device=dev)
+            for i in range(3):
+                z.zipvl_decode(ddesc, qs[i % n_rot], None, None, kcache, vcache, off, capt, seq, max_len,
+                               out=out, ws=ws, status=st)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for i in range(steps):
+                z.zipvl_decode(ddesc, qs[i % n_rot], kn[i % n_rot], vn[i % n_rot], kcache, vcache, off,
+                               capt, seq, max_len, out=out, ws=ws, status=st)
+            e1.record()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1) / steps
+            z.zipvl_decode(ddesc, qs[0], None, None, kcache, vcache, off, capt, seq, max_len, out=out, ws=ws, status=st)
+            torch.cuda.synchronize()
+            b_chk = int(np.argmin(lens))
+            o0, n_rows = int(off[b_chk].item()), int(seq[b_chk].item())
+            ko = kcache[o0:o0 + n_rows * row].float().cpu().numpy()
+            vo = vcache[o0:o0 + n_rows * row].float().cpu().numpy()
+            ref = oracle.decode_step(qs[0][b_chk:b_chk + 1].float().cpu().numpy(), None, None, ko, vo,
+                                     np.zeros(1, np.int64), np.array([n_rows], np.int32), Hkv)
+            dd = np.abs(out[b_chk:b_chk + 1].float().cpu().numpy().astype(np.float64) - ref)
+            tokens = sum(lens) + B * (steps + 1) / 2.0
+            gbs = tokens * row * 4 / (ms * 1e-3) / 1e9
+            res[name] = {"ms_per_step": ms, "tok_s": B / (ms * 1e-3), "hbm_gbs": gbs,
+                         "frac_of_hbm_peak": gbs / peaks["hbm"], "device_status_word": int(st.item()),
+                         "check": {"checked": bool(dd.max() <= 2e-2 and dd.mean() <= 2e-3), "request": b_chk,
+                                   "rows": n_rows, "max_abs": float(dd.max()), "mean_abs": float(dd.mean())}}
+    finally:
+        if prev is None:
+            os.environ.pop("ZIPVL_DECODE_KERNEL", None)
+        else:
+            os.environ["ZIPVL_DECODE_KERNEL"] = prev
+    res["speedup_vs_cuda_core"] = res["cuda_core"]["ms_per_step"] / res["tensor_core"]["ms_per_step"]
+    return res
+
+
 def run_ours(args, rank, world, local):
     import paper_2410_08584_b200 as z
     from paper_2410_08584_b200 import replicas
@@ -841,6 +907,13 @@ def run_ours(args, rank, world, local):
         except Exception as e:  # report, never hide
             dec = {"error": repr(e)}
 
+    dec_gqa = None
+    if args.decode_steps > 0:
+        try:
+            dec_gqa = decode_gqa_benchmark(z, dev, peaks, steps=min(64, args.decode_steps))
+        except Exception as e:  # report, never hide
+            dec_gqa = {"error": repr(e)}
+
     batched = None
     if not args.no_batched:
         try:
@@ -913,7 +986,7 @@ def run_ours(args, rank, world, local):
         "graph_replay_ms_per_step": graph_ms,
         "prefill_ms": float(call_ms[0] + call_ms[1] + call_ms[2]),
         "prefill_tflops_selected": flops / (float(call_ms[0] + call_ms[1] + call_ms[2]) * 1e-3) / 1e12,
-        "roofline": roof, "other_kernels": others, "decode": dec, "batched": batched, "kv_quant": quant, "stack": stack, "long_video": video, "library_context": context,
+        "roofline": roof, "other_kernels": others, "decode": dec, "decode_gqa": dec_gqa, "batched": batched, "kv_quant": quant, "stack": stack, "long_video": video, "library_context": context,
         "cpu_baseline": cpu,
         "e2e": {"value": e2e_ms / world, "unit": "ms", "h2d_bytes_per_step": int(h2d),
                 "d2h_bytes_per_step": int(d2h),
