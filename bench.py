@@ -650,13 +650,13 @@ def decode_benchmark(z, dev, steps, peaks, B=16, ctx_max=32768):
     return res
 
 
-def decode_gqa_benchmark(z, dev, peaks, steps=64, B=16, Hq=28, Hkv=4, d=128):
+def decode_gqa_benchmark(z, dev, peaks, steps=64, B=16, Hq=28, Hkv=4, d=128, len_max=30000):
     """Grouped-query decode (the long-video model's head shape: 28 query heads on 4 kv heads) on kept
     caches of 6K-30K rows: the tensor-core kernel (default from three query heads per kv head) next to
     the CUDA-core kernel, which ZIPVL_DECODE_KERNEL selects; one request checked against the oracle."""
     import oracle
     g = torch.Generator().manual_seed(BASE_SEED + 6)
-    lens = torch.randint(6000, 30001, (B,), generator=g).tolist()
+    lens = torch.randint(len_max // 5, len_max + 1, (B,), generator=g).tolist()
     row = Hkv * d
     caps = [n + steps + 1 for n in lens]
     gd = torch.Generator(device=dev).manual_seed(BASE_SEED + 6)
@@ -901,7 +901,7 @@ def run_ours(args, rank, world, local):
         o["frac_of_hbm_peak"] = o["gbs"] / peaks["hbm"]
 
     dec = None
-    if args.decode_steps > 0:
+    if args.decode_steps > 0 and not args.only_gqa_decode:
         try:
             dec = decode_benchmark(z, dev, args.decode_steps, peaks, args.decode_batch, args.decode_ctx_max)
         except Exception as e:  # report, never hide
@@ -910,7 +910,8 @@ def run_ours(args, rank, world, local):
     dec_gqa = None
     if args.decode_steps > 0:
         try:
-            dec_gqa = decode_gqa_benchmark(z, dev, peaks, steps=min(64, args.decode_steps))
+            dec_gqa = decode_gqa_benchmark(z, dev, peaks, steps=min(64, args.decode_steps), B=args.gqa_batch,
+                                           len_max=args.gqa_len_max)
         except Exception as e:  # report, never hide
             dec_gqa = {"error": repr(e)}
 
@@ -1005,6 +1006,11 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--decode-steps", type=int, default=256)
     ap.add_argument("--decode-batch", type=int, default=16, help="requests in the batched-decode leg")
+    ap.add_argument("--gqa-batch", type=int, default=16, help="requests in the grouped-query decode leg")
+    ap.add_argument("--gqa-len-max", type=int, default=30000,
+                    help="longest kept cache of the grouped-query decode leg (smaller = a light profiling case)")
+    ap.add_argument("--only-gqa-decode", action="store_true",
+                    help="of the two decode legs run only the grouped-query one (profiling)")
     ap.add_argument("--decode-ctx-max", type=int, default=32768,
                     help="largest context of the batched-decode leg (smaller = a light profiling case)")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -296,10 +296,12 @@ zipvl_status zipvl_sparse_prefill_batch(const zipvl_layer *layer, const zipvl_ba
  * its cache is read or written, its output is zeros, its length stays) and
  * reported as ZIPVL_DEV_BAD_INDEX.  The call enqueues two kernels (the second merges the cache chunks).
  * Query heads per kv head (Hq / Hkv): up to 8 for any dtype and head_dim; up to 32 in 16-bit
- * storage at head_dim 128, where from 3 on the step runs on the tensor cores (the query heads of
- * a kv head are the rows of an MMA tile, so grouped-query attention stays bound by HBM instead of
- * by multiply-adds).  Same results contract either way; ZIPVL_DECODE_KERNEL=simt|tc in the
- * environment forces one of the two kernels where both apply.
+ * storage at head_dim 128, where grouped heads run on the tensor cores (the query heads of a kv
+ * head are the rows of an MMA tile, so grouped-query attention stays bound by HBM instead of by
+ * multiply-adds): one CTA per chunk of a request's cache for small problems, a persistent launch
+ * (one CTA per SM over an equal share of all key/value tiles) for large ones.  Same results
+ * contract on every path; ZIPVL_DECODE_KERNEL=simt|tc|tcp in the environment forces the
+ * CUDA-core, the chunked or the persistent tensor-core kernel where it applies.
  */
 zipvl_status zipvl_decode(const zipvl_decode_desc *desc, const void *q, const void *k_new,
                           const void *v_new, void *k_cache, void *v_cache,

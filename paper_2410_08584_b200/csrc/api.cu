@@ -97,7 +97,7 @@ size_t zipvl_workspace_bytes(int32_t op, const zipvl_layer *layer, int32_t n_pro
         case ZIPVL_OP_COMPACT_KV: return 256;
         case ZIPVL_OP_DECODE:
             if (batch < 1) return 0;
-            return align256(decode_ws_bytes(batch, a.Hq, a.D, a.L));
+            return align256(decode_ws_bytes(batch, a.Hq, a.D, a.L, a.Hkv, layer->dtype));
     }
     return 0;
 }
@@ -247,7 +247,7 @@ zipvl_status zipvl_decode(const zipvl_decode_desc *d, const void *q, const void 
         return fail(ZIPVL_ERR_INVALID_ARG, "zipvl_decode: softmax_scale");
     if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(out) || !aligned16(ws))
         return fail(ZIPVL_ERR_INVALID_ARG, "zipvl_decode: tensors must be 16-byte aligned");
-    const size_t need = align256(decode_ws_bytes(d->batch, d->n_q_heads, d->head_dim, max_len));
+    const size_t need = align256(decode_ws_bytes(d->batch, d->n_q_heads, d->head_dim, max_len, d->n_kv_heads, d->dtype));
     if (ws_bytes < need) return fail(ZIPVL_ERR_WORKSPACE, "zipvl_decode: workspace %zu < %zu", ws_bytes, need);
     const float scale = d->softmax_scale > 0.f ? d->softmax_scale : 1.0f / sqrtf((float)d->head_dim);
     return launch_decode(*d, scale * kLog2e, q, k_new, v_new, k_cache, v_cache, cache_off, capacity,
@@ -469,7 +469,7 @@ zipvl_status zipvl_layer_step_host(const zipvl_layer *layer, const void *q, cons
     size_t ws_b = ws_score > ws_pf ? ws_score : ws_pf;
     if (ws_b < select_ws_bytes()) ws_b = select_ws_bytes();
     // the decode step runs on the cache this call has just compacted: capacity L + 1 rows
-    const size_t ws_dec = with_decode ? align256(decode_ws_bytes(1, a.Hq, a.D, a.L + 1)) : 0;
+    const size_t ws_dec = with_decode ? align256(decode_ws_bytes(1, a.Hq, a.D, a.L + 1, a.Hkv, layer->dtype)) : 0;
     if (ws_b < ws_dec) ws_b = ws_dec;
     const size_t qn_b = (size_t)a.Hq * a.D * eb, kn_b = (size_t)a.Hkv * a.D * eb;
     // one stream-ordered allocation carved into pieces

@@ -150,20 +150,34 @@ struct PageArgs {
     int stride, shift, n_pages;
 };
 
-size_t decode_ws_bytes(int B, int Hq, int D, int max_len);
+// (Hkv and dtype decide whether the grouped-query tensor-core kernel, which leaves more partials,
+// may run: 0 / -1 = the CUDA-core layout)
+size_t decode_ws_bytes(int B, int Hq, int D, int max_len, int Hkv = 0, int dtype = -1);
 int decode_chunk_rows(int B, int Hq, int max_len);
 size_t decode_partial_bytes(int B, int Hq, int D, int max_len);
+// used != nullptr: used[b * (Hq / group) + hq / group] of the n_chunks slots hold a partial
 zipvl_status launch_decode_merge(int dtype, int D, int Hq, int B, int chunk, int n_chunks, const float *ws,
-                                 const int *lens, int32_t *seq_lens, void *out, cudaStream_t st);
-// Grouped-query decode on the tensor cores (decode_tc.cu): 16-bit storage, head_dim 128, 2 to 32
-// query heads per kv head.  Leaves per-chunk partials and the (length, appended) pairs in the
-// layout of the kernels in decode.cu and returns the chunk it used; the caller launches the merge.
+                                 const int *lens, int32_t *seq_lens, void *out, cudaStream_t st,
+                                 const int *used = nullptr, int group = 1);
+// Grouped-query decode on the tensor cores: 16-bit storage, head_dim 128, 2 to 32 query heads per
+// kv head.  Two kernels that leave partials in the layout of the kernels in decode.cu and the
+// (length, appended) pairs in lens[]; the caller launches the merge.
+//   decode_tc.cu             one CTA per chunk of a (request, kv head): one partial per chunk, returns
+//                            the chunk it used (never smaller than min_chunk);
+//   decode_tc_persistent.cu  one CTA per SM over an equal share of all tiles (large batches): four
+//                            partials per CTA and (request, kv head), n_slots per (request, query
+//                            head), the number in use per (request, kv head) in used[].
 bool decode_tc_supported(const zipvl_decode_desc &d);
 zipvl_status launch_decode_tc(const zipvl_decode_desc &d, float scale_log2, const void *q,
                               const void *k_new, const void *v_new, void *k_cache, void *v_cache,
                               const int64_t *cache_off, PageArgs pg, const int32_t *capacity,
                               int32_t *seq_lens, int max_len, int min_chunk, float *partials, int *lens,
                               int32_t *status_word, cudaStream_t st, int *chunk_out);
+zipvl_status launch_decode_tcp(const zipvl_decode_desc &d, float scale_log2, const void *q,
+                               const void *k_new, const void *v_new, void *k_cache, void *v_cache,
+                               const int64_t *cache_off, PageArgs pg, const int32_t *capacity,
+                               int32_t *seq_lens, int max_len, int n_slots, float *partials, int *lens,
+                               int *used, int32_t *status_word, cudaStream_t st);
 zipvl_status launch_decode(const zipvl_decode_desc &d, float scale_log2, const void *q,
                            const void *k_new, const void *v_new, void *k_cache, void *v_cache,
                            const int64_t *cache_off, const int32_t *capacity, int32_t *seq_lens,

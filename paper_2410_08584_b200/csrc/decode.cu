@@ -277,22 +277,25 @@ constexpr int kMergeLanes = 8;
 template <typename T, int D>
 __global__ void __launch_bounds__(256)
 decode_merge_kernel(int Hq, int chunk, int n_chunks, const float *__restrict__ ws,
-                    const int *__restrict__ lens, int32_t *__restrict__ seq_lens, T *__restrict__ out) {
+                    const int *__restrict__ lens, int32_t *__restrict__ seq_lens, T *__restrict__ out,
+                    const int *__restrict__ used, int group) {
     grid_launch_dependents();
-    grid_dependency_wait(ws, lens, seq_lens);
+    grid_dependency_wait(ws, lens, seq_lens, used);
     const int b = blockIdx.y;
     const int t = (blockIdx.x * 256 + threadIdx.x) / kMergeLanes;       // (head, channel) of this lane group
     const int part = threadIdx.x % kMergeLanes;
     const bool live = t < Hq * D;
     const int hq = live ? t / D : 0, c = live ? t % D : 0;
     const float *src = ws + ((long long)b * Hq + hq) * n_chunks * (D + 2);
+    // the tensor-core kernel fills only the first used[request, kv head] slots of a head
+    const int n_used = used ? min(n_chunks, max(0, used[b * (Hq / group) + hq / group])) : n_chunks;
     float M = -INFINITY, Ls = 0.f, Os = 0.f;
-    for (int i0 = part; i0 < n_chunks; i0 += 8 * kMergeLanes) {
+    for (int i0 = part; i0 < n_used; i0 += 8 * kMergeLanes) {
         float mi[8], li[8], oi[8];
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
             const int i = i0 + u * kMergeLanes;
-            const bool in = live && i < n_chunks;
+            const bool in = live && i < n_used;
             const float *p = src + (long long)(in ? i : 0) * (D + 2);
             mi[u] = in ? __ldcg(p) : -INFINITY;
             li[u] = in ? __ldcg(p + 1) : 0.f;
@@ -338,12 +341,28 @@ int decode_chunk(int B, int Hq, int max_len) {
     return c;
 }
 
-size_t partial_bytes(int B, int Hq, int D, int max_len) {
+// partials per (request, query head) in the workspace: one per chunk for the CUDA-core kernel and
+// the chunked tensor-core kernel; the persistent tensor-core kernel cuts the work by tiles (a
+// request of c chunks' worth of tiles may be shared by c + 1 CTAs) and leaves four partials per CTA
+int partial_slots(int B, int Hq, int max_len, bool tc) {
     const int chunk = decode_chunk(B, Hq, max_len);
-    const size_t n_chunks = (max_len + chunk - 1) / chunk;
-    return ((size_t)B * Hq * n_chunks * (D + 2) * sizeof(float) + 255) & ~(size_t)255;
+    const int n_chunks = (max_len + chunk - 1) / chunk;
+    return tc ? 4 * (n_chunks + 1) : n_chunks;
 }
-size_t counter_bytes(int B, int) { return (size_t)(2 * B) * sizeof(int); }   // (length, appended) per request
+bool tc_shape(int Hq, int Hkv, int D, int dtype) {
+    if (Hkv < 1 || Hq % Hkv) return false;
+    const zipvl_decode_desc d = {1, Hq, Hkv, D, dtype, 0.f};
+    return decode_tc_supported(d);
+}
+
+size_t partial_bytes(int B, int Hq, int D, int max_len, bool tc = false) {
+    if (tc) return ((size_t)B * Hq * partial_slots(B, Hq, max_len, true) * (D + 2) * sizeof(float) + 255) & ~(size_t)255;
+    const int chunk = decode_chunk(B, Hq, max_len);
+    const size_t n_slots = (max_len + chunk - 1) / chunk;
+    return ((size_t)B * Hq * n_slots * (D + 2) * sizeof(float) + 255) & ~(size_t)255;
+}
+// (length, appended) per request, and for the tensor-core kernel the slots in use per (request, kv head)
+size_t counter_bytes(int B, int Hq) { return (size_t)(2 * B + B * Hq) * sizeof(int); }
 
 template <typename T, int D>
 zipvl_status run(const zipvl_decode_desc &d, float scale_log2, const void *q, const void *k_new,
@@ -377,7 +396,8 @@ zipvl_status run(const zipvl_decode_desc &d, float scale_log2, const void *q, co
 #undef ZIPVL_DEC_P
     if (le == cudaSuccess)
         le = launch_dependent(decode_merge_kernel<T, D>, dim3((Hq * D * kMergeLanes + 255) / 256, B), dim3(256), 0, st, Hq,
-                              chunk, n_chunks, (const float *)wsf, (const int *)lens, seq_lens, (T *)out);
+                              chunk, n_chunks, (const float *)wsf, (const int *)lens, seq_lens, (T *)out,
+                              (const int *)nullptr, 1);
     if (le != cudaSuccess) return fail(ZIPVL_ERR_CUDA, "zipvl_decode: launch: %s", cudaGetErrorString(le));
     count_launches(2);
     return check_launch("zipvl_decode");
@@ -390,11 +410,12 @@ zipvl_status run(const zipvl_decode_desc &d, float scale_log2, const void *q, co
 int decode_chunk_rows(int B, int Hq, int max_len) { return decode_chunk(B, Hq, max_len); }
 size_t decode_partial_bytes(int B, int Hq, int D, int max_len) { return partial_bytes(B, Hq, D, max_len); }
 zipvl_status launch_decode_merge(int dtype, int D, int Hq, int B, int chunk, int n_chunks, const float *ws,
-                                 const int *lens, int32_t *seq_lens, void *out, cudaStream_t st) {
+                                 const int *lens, int32_t *seq_lens, void *out, cudaStream_t st,
+                                 const int *used, int group) {
     cudaError_t le = cudaErrorInvalidValue;
     const dim3 grid((Hq * D * kMergeLanes + 255) / 256, B);
 #define ZIPVL_MERGE(T_, D_) \
-    le = launch_dependent(decode_merge_kernel<T_, D_>, grid, dim3(256), 0, st, Hq, chunk, n_chunks, ws, lens, seq_lens, (T_ *)out)
+    le = launch_dependent(decode_merge_kernel<T_, D_>, grid, dim3(256), 0, st, Hq, chunk, n_chunks, ws, lens, seq_lens, (T_ *)out, used, group)
     if (dtype == ZIPVL_BF16 && D == 128) ZIPVL_MERGE(__nv_bfloat16, 128);
     else if (dtype == ZIPVL_BF16 && D == 96) ZIPVL_MERGE(__nv_bfloat16, 96);
     else if (dtype == ZIPVL_BF16 && D == 64) ZIPVL_MERGE(__nv_bfloat16, 64);
@@ -407,8 +428,8 @@ zipvl_status launch_decode_merge(int dtype, int D, int Hq, int B, int chunk, int
     return ZIPVL_OK;
 }
 
-size_t decode_ws_bytes(int B, int Hq, int D, int max_len) {
-    return partial_bytes(B, Hq, D, max_len) + counter_bytes(B, Hq);
+size_t decode_ws_bytes(int B, int Hq, int D, int max_len, int Hkv, int dtype) {
+    return partial_bytes(B, Hq, D, max_len, tc_shape(Hq, Hkv, D, dtype)) + counter_bytes(B, Hq);
 }
 
 namespace {
@@ -418,25 +439,43 @@ zipvl_status dispatch_decode(const zipvl_decode_desc &d, float scale_log2, const
                              int32_t *seq_lens, int max_len, void *out, void *ws,
                              int32_t *status_word, cudaStream_t st) {
     // Grouped-query attention in 16-bit storage at head_dim 128 runs on the tensor cores from
-    // three query heads per kv head on: there the CUDA-core kernel is bound by its multiply-adds
-    // (0.51 of the HBM copy rate at four heads per kv head, 0.27 at seven, against 0.76 here;
-    // at two it still reaches 0.81).  ZIPVL_DECODE_KERNEL=simt|tc overrides the choice
-    // (measurements, tests).
+    // two query heads per kv head on: there the CUDA-core kernel is bound by its multiply-adds
+    // (0.51 of the HBM copy rate at four heads per kv head, 0.27 at seven; at two it still reaches
+    // 0.81).  Of the two tensor-core kernels the persistent one takes the large problems (from
+    // about 14 key/value tiles per SM on it is 5 to 10 % faster: no CTA prologue between work
+    // items); below that the launch of one CTA per chunk is quicker (fewer partials to merge,
+    // shorter CTAs).  ZIPVL_DECODE_KERNEL=simt|tc|tcp overrides the choice (measurements, tests).
     {
         const char *env = getenv("ZIPVL_DECODE_KERNEL");
         const int G = d.n_q_heads / d.n_kv_heads;
-        const bool want_tc = env ? !strcmp(env, "tc") : G >= 3;
-        if (decode_tc_supported(d) && (want_tc || G > 8)) {
+        const long long tiles = (long long)d.batch * d.n_kv_heads * ((max_len + 127) / 128);
+        // (two query heads per kv head: the CUDA-core kernel is the faster one on large batches,
+        // 0.81 against 0.74 of the copy rate, the chunked tensor-core kernel on small ones)
+        const bool want_simt = env ? !strcmp(env, "simt") : (G < 3 && tiles >= 2000);
+        if (decode_tc_supported(d) && (!want_simt || G > 8)) {
             const int B = d.batch, Hq = d.n_q_heads, D = d.head_dim;
+            const bool persistent = env && !strcmp(env, "tcp") ? true
+                                    : (env && !strcmp(env, "tc") ? false : tiles >= 2000);
             float *wsf = reinterpret_cast<float *>(ws);
-            int *lens = reinterpret_cast<int *>(reinterpret_cast<char *>(ws) + partial_bytes(B, Hq, D, max_len));
-            int chunk = 0;
-            const zipvl_status s = launch_decode_tc(d, scale_log2, q, k_new, v_new, k_cache, v_cache, cache_off,
-                                                    pg, capacity, seq_lens, max_len, decode_chunk(B, Hq, max_len),
-                                                    wsf, lens, status_word, st, &chunk);
-            if (s != ZIPVL_OK) return s;
-            const zipvl_status sm = launch_decode_merge(d.dtype, D, Hq, B, chunk, (max_len + chunk - 1) / chunk,
-                                                        wsf, lens, seq_lens, out, st);
+            int *lens = reinterpret_cast<int *>(reinterpret_cast<char *>(ws) + partial_bytes(B, Hq, D, max_len, true));
+            int *used = lens + 2 * B;
+            int chunk = decode_chunk(B, Hq, max_len);
+            zipvl_status sm;
+            if (persistent) {
+                const int n_slots = partial_slots(B, Hq, max_len, true);    // as the workspace was sized
+                const zipvl_status s = launch_decode_tcp(d, scale_log2, q, k_new, v_new, k_cache, v_cache,
+                                                         cache_off, pg, capacity, seq_lens, max_len, n_slots, wsf,
+                                                         lens, used, status_word, st);
+                if (s != ZIPVL_OK) return s;
+                sm = launch_decode_merge(d.dtype, D, Hq, B, chunk, n_slots, wsf, lens, seq_lens, out, st, used, G);
+            } else {
+                const zipvl_status s = launch_decode_tc(d, scale_log2, q, k_new, v_new, k_cache, v_cache, cache_off,
+                                                        pg, capacity, seq_lens, max_len, chunk, wsf, lens,
+                                                        status_word, st, &chunk);
+                if (s != ZIPVL_OK) return s;
+                sm = launch_decode_merge(d.dtype, D, Hq, B, chunk, (max_len + chunk - 1) / chunk, wsf, lens,
+                                         seq_lens, out, st);
+            }
             return sm != ZIPVL_OK ? sm : check_launch("zipvl_decode");
         }
         if (G > 8) return fail(ZIPVL_ERR_UNSUPPORTED, "decode: %d query heads per kv head", G);
@@ -531,7 +570,7 @@ extern "C" zipvl_status zipvl_decode_noalloc(const zipvl_decode_desc *d, const v
         return fail(ZIPVL_ERR_INVALID_ARG, "%s: softmax_scale", who);
     if (((uintptr_t)q | (uintptr_t)k_cache | (uintptr_t)v_cache | (uintptr_t)out) & 15u)
         return fail(ZIPVL_ERR_INVALID_ARG, "%s: tensors must be 16-byte aligned", who);
-    const size_t need = decode_ws_bytes(d->batch, d->n_q_heads, d->head_dim, max_len);
+    const size_t need = decode_ws_bytes(d->batch, d->n_q_heads, d->head_dim, max_len, d->n_kv_heads, d->dtype);
     if (need > kNoAllocScratchBytes)
         return fail(ZIPVL_ERR_WORKSPACE,
                     "%s: batch %d x %d heads x max_len %d needs %zu bytes of scratch, the built-in "
@@ -582,7 +621,7 @@ extern "C" zipvl_status zipvl_decode_paged(const zipvl_decode_desc *d, const voi
         return fail(ZIPVL_ERR_INVALID_ARG, "%s: softmax_scale", who);
     if (((uintptr_t)q | (uintptr_t)k_pages | (uintptr_t)v_pages | (uintptr_t)out | (uintptr_t)ws) & 15u)
         return fail(ZIPVL_ERR_INVALID_ARG, "%s: tensors must be 16-byte aligned", who);
-    const size_t need = (decode_ws_bytes(d->batch, d->n_q_heads, d->head_dim, max_len) + 255) & ~(size_t)255;
+    const size_t need = (decode_ws_bytes(d->batch, d->n_q_heads, d->head_dim, max_len, d->n_kv_heads, d->dtype) + 255) & ~(size_t)255;
     if (ws_bytes < need) return fail(ZIPVL_ERR_WORKSPACE, "%s: workspace %zu < %zu", who, ws_bytes, need);
     const float scale = d->softmax_scale > 0.f ? d->softmax_scale : 1.0f / sqrtf((float)d->head_dim);
     return dispatch_decode(*d, scale * kLog2e, q, k_new, v_new, k_pages, v_pages, nullptr,

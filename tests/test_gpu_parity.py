@@ -769,10 +769,34 @@ def test_decode_parity(zipvl, lens, Hq, Hkv, d, dtype):
     assert st.item() & zipvl.DEV_CAPACITY and np.array_equal(seq_d.cpu().numpy(), seq_o)
 
 
+@pytest.mark.parametrize("lens,Hq,Hkv,dtype", [
+    ([513, 40, 2000], 14, 2, torch.bfloat16),
+    ([5000, 129, 0, 3000, 1], 28, 4, torch.bfloat16),
+    ([2100, 640], 32, 2, torch.float16),
+])
+def test_decode_parity_on_the_persistent_kernel(zipvl, monkeypatch, lens, Hq, Hkv, dtype):
+    """The decode parity test (three steps with appends, a step without, a full cache) with the
+    persistent tensor-core kernel forced: by default it only takes large batches."""
+    monkeypatch.setenv("ZIPVL_DECODE_KERNEL", "tcp")
+    test_decode_parity(zipvl, lens, Hq, Hkv, 128, dtype)
+
+
+@pytest.mark.parametrize("lens,Hq,Hkv,dtype,page_rows", [
+    ([513, 40, 2000, 0], 16, 4, torch.bfloat16, 16),
+    ([3000, 100], 28, 4, torch.float16, 256),
+])
+def test_paged_decode_parity_on_the_persistent_kernel(zipvl, monkeypatch, lens, Hq, Hkv, dtype, page_rows):
+    monkeypatch.setenv("ZIPVL_DECODE_KERNEL", "tcp")
+    test_paged_decode_parity(zipvl, lens, Hq, Hkv, 128, dtype, page_rows)
+
+
 @pytest.mark.parametrize("kernel,lens,Hq,Hkv", [
     ("tc", [700, 130, 2600], 8, 4),        # two query heads per kv head: the CUDA-core kernel by default
     ("simt", [700, 130, 2600], 14, 2),     # seven: the tensor-core kernel by default
     ("tc", [4000], 64, 2),                 # thirty-two, several tiles per CTA
+    ("tcp", [700, 130, 2600], 14, 2),      # the persistent kernel (large batches by default)
+    ("tcp", [4000, 129], 64, 2),           # thirty-two heads: one set of query rows
+    ("tcp", [30000, 9000, 128, 0, 5000], 28, 4),   # long runs of tiles per CTA, an empty request
 ])
 def test_decode_kernel_choice_can_be_forced_and_both_match_the_oracle(zipvl, monkeypatch, kernel, lens, Hq, Hkv):
     """ZIPVL_DECODE_KERNEL picks the grouped-query decode kernel; either choice has to match the
@@ -787,7 +811,7 @@ def test_decode_kernel_choice_can_be_forced_and_both_match_the_oracle(zipvl, mon
     ref = oracle.decode_step(to_np(q), None, None, kc.float().numpy(), vc.float().numpy(), off.numpy(),
                              np.array(lens, np.int32), Hkv)
     outs = {}
-    for which in (kernel, "simt" if kernel == "tc" else "tc"):
+    for which in (kernel, "simt" if kernel != "simt" else "tc"):
         if Hq // Hkv > 8 and which == "simt":
             continue                        # more than eight query heads per kv head: tensor cores only
         monkeypatch.setenv("ZIPVL_DECODE_KERNEL", which)
@@ -798,7 +822,8 @@ def test_decode_kernel_choice_can_be_forced_and_both_match_the_oracle(zipvl, mon
         check_attention(to_np(a), ref, dtype)
         outs[which] = a
     if len(outs) == 2:
-        check_attention(to_np(outs["tc"]), to_np(outs["simt"]).astype(np.float64), dtype)
+        a, b = list(outs.values())
+        check_attention(to_np(a), to_np(b).astype(np.float64), dtype)
 
 
 @pytest.mark.parametrize("lens,Hq,Hkv,d,dtype,page_rows", [
