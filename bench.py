@@ -677,7 +677,12 @@ def decode_gqa_benchmark(z, dev, peaks, steps=64, B=16, Hq=28, Hkv=4, d=128, len
     prev = os.environ.get("ZIPVL_DECODE_KERNEL")
     try:
         for name in ("tensor_core", "cuda_core"):
-            os.environ["ZIPVL_DECODE_KERNEL"] = "tc" if name == "tensor_core" else "simt"
+            # the library's own choice of tensor-core kernel (chunked or persistent, by problem size)
+            # against the CUDA-core kernel forced
+            if name == "tensor_core":
+                os.environ.pop("ZIPVL_DECODE_KERNEL", None)
+            else:
+                os.environ["ZIPVL_DECODE_KERNEL"] = "simt"
             seq = torch.tensor(lens, dtype=torch.int32, device=dev)
             st = torch.zeros(1, dtype=torch.int32, device=dev)
             for i in range(3):
