@@ -595,10 +595,12 @@ def test_a_bounded_wait_that_runs_out_is_reported_and_the_context_survives(zipvl
     assert r["status"] == 0 and r["k"] >= 1
 
 
-def test_decode_skips_requests_with_impossible_lengths_or_offsets(zipvl):
+@pytest.mark.parametrize("kernel", ["simt", "tc", "tcp"])
+def test_decode_skips_requests_with_impossible_lengths_or_offsets(zipvl, monkeypatch, kernel):
     """seq_lens < 0, seq_lens > capacity and a cache offset off the 16-byte grid: the request
     is skipped (zero output, cache and length untouched) and reported; the other requests of
     the batch are served as usual.  All buffers are in range, so nothing can fault."""
+    monkeypatch.setenv("ZIPVL_DECODE_KERNEL", kernel)      # the CUDA-core kernel and both tensor-core ones
     lens, Hq, Hkv, d = [40, 300, 77, 130], 4, 2, 128
     B = len(lens)
     kc, vc, off, cap = build_caches(lens, Hkv, d, torch.bfloat16, 4, seed=8)
