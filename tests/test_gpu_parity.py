@@ -1022,3 +1022,61 @@ def test_layer_step_replays_from_a_cuda_graph(zipvl):
                     got, want = got[:n_rows], want[:n_rows]
                 assert torch.equal(got, want), j
     assert int(st.item()) == 0
+
+
+@pytest.mark.parametrize("kernel", ["tc", "tcp"])
+def test_grouped_query_decode_steps_replay_from_a_cuda_graph(zipvl, monkeypatch, kernel):
+    """Four decode steps with appends on grouped query heads, captured once into a CUDA graph
+    (lengths live on the device, each step is a programmatic dependent of the one before) and
+    replayed from reset lengths: the replays must equal eager execution bit for bit -- outputs,
+    lengths and the appended cache rows."""
+    monkeypatch.setenv("ZIPVL_DECODE_KERNEL", kernel)
+    lens, Hq, Hkv, d, steps = [700, 129, 2600, 1], 14, 2, 128, 4
+    B = len(lens)
+    kc, vc, off, cap = build_caches(lens, Hkv, d, torch.bfloat16, steps, seed=77)
+    g = torch.Generator().manual_seed(78)
+    qs = torch.randn(steps, B, Hq, d, generator=g).bfloat16().to(DEV)
+    kn = torch.randn(steps, B, Hkv, d, generator=g).bfloat16().to(DEV)
+    vn = torch.randn(steps, B, Hkv, d, generator=g).bfloat16().to(DEV)
+    desc = zipvl.zipvl_decode_desc(B, Hq, Hkv, d, zipvl.ZIPVL_BF16, 0.0)
+    max_len = max(lens) + steps
+    dl = zipvl.zipvl_layer(max_len, Hq, Hkv, d, zipvl.ZIPVL_BF16, 0, 0, 0, 0.0, 0)
+    ws = zipvl.workspace(zipvl.zipvl_workspace_bytes(zipvl.OP_DECODE, dl, 0, B), DEV)
+    kc_d, vc_d, off_d, cap_d = kc.to(DEV), vc.to(DEV), off.to(DEV), cap.to(DEV)
+    seq0 = torch.tensor(lens, dtype=torch.int32, device=DEV)
+    seq = seq0.clone()
+    outs = torch.empty(steps, B, Hq, d, dtype=torch.bfloat16, device=DEV)
+    st = status_word()
+
+    def run():
+        for s in range(steps):
+            zipvl.zipvl_decode(desc, qs[s], kn[s], vn[s], kc_d, vc_d, off_d, cap_d, seq, max_len,
+                               out=outs[s], ws=ws, status=st)
+
+    run()
+    torch.cuda.synchronize()
+    want = (outs.clone(), seq.clone(), kc_d.clone(), vc_d.clone())
+    # the eager run against the oracle, step by step
+    ko, vo, seqo = to_np(kc).copy(), to_np(vc).copy(), np.array(lens, np.int32)
+    for s in range(steps):
+        ref = oracle.decode_step(to_np(qs[s].cpu()), to_np(kn[s].cpu()), to_np(vn[s].cpu()), ko, vo,
+                                 off.numpy(), seqo, Hkv)
+        check_attention(to_np(want[0][s].cpu()), ref, torch.bfloat16)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        seq.copy_(seq0)
+        run()                                    # warm-up on the capture stream
+        seq.copy_(seq0)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            run()
+    torch.cuda.current_stream().wait_stream(side)
+    for rep in range(3):
+        seq.copy_(seq0)
+        outs.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(outs, want[0]) and torch.equal(seq, want[1])
+        assert torch.equal(kc_d, want[2]) and torch.equal(vc_d, want[3])
+    assert int(st.item()) == 0
