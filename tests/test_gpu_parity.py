@@ -1080,3 +1080,44 @@ def test_grouped_query_decode_steps_replay_from_a_cuda_graph(zipvl, monkeypatch,
         assert torch.equal(outs, want[0]) and torch.equal(seq, want[1])
         assert torch.equal(kc_d, want[2]) and torch.equal(vc_d, want[3])
     assert int(st.item()) == 0
+
+
+@pytest.mark.parametrize("kernel", ["tc", "tcp"])
+@pytest.mark.parametrize("seed", [0, 1, 2, 3])
+def test_grouped_query_decode_random_batches(zipvl, monkeypatch, kernel, seed):
+    """Random ragged batches on the tensor-core decode kernels: empty and one-row requests next to
+    requests of several tiles, group sizes from 3 to 16, with and without a new token, two steps
+    each, against the oracle.  (Short and long work items side by side are what the persistent
+    kernel's segment hand-over has to get right.)"""
+    monkeypatch.setenv("ZIPVL_DECODE_KERNEL", kernel)
+    rng = np.random.default_rng(1000 + seed)
+    for trial in range(3):
+        G = int(rng.choice([3, 4, 7, 8, 16]))
+        Hkv = int(rng.choice([1, 2, 4]))
+        Hq, d = G * Hkv, 128
+        B = int(rng.integers(1, 7))
+        lens = [int(x) for x in rng.choice([0, 1, 5, 127, 128, 129, 300, 777, 1500, 2600, 4100], size=B)]
+        dtype = torch.bfloat16 if trial % 2 == 0 else torch.float16
+        code = zipvl.ZIPVL_BF16 if dtype == torch.bfloat16 else zipvl.ZIPVL_F16
+        kc, vc, off, cap = build_caches(lens, Hkv, d, dtype, 2, seed=seed * 10 + trial)
+        g = torch.Generator().manual_seed(seed * 100 + trial)
+        desc = zipvl.zipvl_decode_desc(B, Hq, Hkv, d, code, 0.0)
+        kc_d, vc_d, off_d, cap_d = kc.to(DEV), vc.to(DEV), off.to(DEV), cap.to(DEV)
+        seq_d = torch.tensor(lens, dtype=torch.int32, device=DEV)
+        ko, vo, seqo = kc.float().numpy().copy(), vc.float().numpy().copy(), np.array(lens, np.int32)
+        st = status_word()
+        max_len = max(lens) + 2
+        for step in range(2):
+            q = torch.randn(B, Hq, d, generator=g).to(dtype)
+            append = bool((seed + trial + step) % 2 == 0)
+            kn = torch.randn(B, Hkv, d, generator=g).to(dtype) if append else None
+            vn = torch.randn(B, Hkv, d, generator=g).to(dtype) if append else None
+            out = zipvl.zipvl_decode(desc, q.to(DEV), None if kn is None else kn.to(DEV),
+                                     None if vn is None else vn.to(DEV), kc_d, vc_d, off_d, cap_d, seq_d,
+                                     max_len, status=st)
+            ref = oracle.decode_step(to_np(q), None if kn is None else to_np(kn),
+                                     None if vn is None else to_np(vn), ko, vo, off.numpy(), seqo, Hkv)
+            check_attention(to_np(out), ref, dtype)
+            assert np.array_equal(seq_d.cpu().numpy(), seqo)
+        assert st.item() == 0
+        assert np.array_equal(kc_d.float().cpu().numpy(), ko) and np.array_equal(vc_d.float().cpu().numpy(), vo)
