@@ -381,9 +381,11 @@ zipvl_status zipvl_decode_quant(const zipvl_decode_desc *desc, const void *q, co
  * batch * n_q_heads * ceil(max_len / chunk) * (head_dim + 2) * 4 bytes must fit
  * in 8 MiB, where chunk is the number of cache rows the library gives one thread
  * block (a power of two from 32 to 512, growing with the problem) -- e.g. batch
- * 16, 32 heads, head_dim 128 fits up to max_len 15872.  Larger problems are
- * refused with ZIPVL_ERR_WORKSPACE and a message; use zipvl_decode with a
- * workspace.
+ * 16, 32 heads, head_dim 128 fits up to max_len 15872.  A shape the grouped-query
+ * tensor-core kernels take (16-bit storage, head_dim 128, 2 to 32 query heads per
+ * kv head) needs 4 * (ceil(max_len / chunk) + 1) such slots per query head plus
+ * 4 bytes per (request, query head).  Larger problems are refused with
+ * ZIPVL_ERR_WORKSPACE and a message; use zipvl_decode with a workspace.
  *
  * The first call on each device looks up the array's device address (with that
  * device current) and caches it for the life of the process; make that first
