@@ -295,8 +295,8 @@ zipvl_status zipvl_sparse_prefill_batch(const zipvl_layer *layer, const zipvl_ba
  * cache_off[b] is not a multiple of 16 bytes, is skipped as a whole (nothing of
  * its cache is read or written, its output is zeros, its length stays) and
  * reported as ZIPVL_DEV_BAD_INDEX.  The call enqueues two kernels (the second merges the cache chunks).
- * Query heads per kv head (Hq / Hkv): up to 8 for any dtype and head_dim; up to 32 in 16-bit
- * storage at head_dim 128, where grouped heads run on the tensor cores (the query heads of a kv
+ * Query heads per kv head (Hq / Hkv): up to 8 for any dtype; up to 32 in 16-bit storage,
+ * where grouped heads run on the tensor cores (the query heads of a kv
  * head are the rows of an MMA tile, so grouped-query attention stays bound by HBM instead of by
  * multiply-adds): one CTA per chunk of a request's cache for small problems, a persistent launch
  * (one CTA per SM over an equal share of all key/value tiles) for large ones.  Same results
@@ -382,8 +382,7 @@ zipvl_status zipvl_decode_quant(const zipvl_decode_desc *desc, const void *q, co
  * in 8 MiB, where chunk is the number of cache rows the library gives one thread
  * block (a power of two from 32 to 512, growing with the problem) -- e.g. batch
  * 16, 32 heads, head_dim 128 fits up to max_len 15872.  A shape the grouped-query
- * tensor-core kernels take (16-bit storage, head_dim 128, 2 to 32 query heads per
- * kv head) needs 4 * (ceil(max_len / chunk) + 1) such slots per query head plus
+ * tensor-core kernels take (16-bit storage, 2 to 32 query heads per kv head) needs 4 * (ceil(max_len / chunk) + 1) such slots per query head plus
  * 4 bytes per (request, query head).  Larger problems are refused with
  * ZIPVL_ERR_WORKSPACE and a message; use zipvl_decode with a workspace.
  *

@@ -237,7 +237,7 @@ zipvl_status zipvl_decode(const zipvl_decode_desc *d, const void *q, const void 
         return fail(ZIPVL_ERR_UNSUPPORTED, "zipvl_decode: head_dim %d (64, 96 or 128)", d->head_dim);
     if (d->n_q_heads / d->n_kv_heads > 8 && !decode_tc_supported(*d))
         return fail(ZIPVL_ERR_UNSUPPORTED, "zipvl_decode: more than 8 query heads per kv head (up to 32 "
-                                           "in 16-bit storage at head_dim 128)");
+                                           "in 16-bit storage)");
     if (!q || !k_cache || !v_cache || !cache_off || !capacity || !seq_lens || !out || !ws)
         return fail(ZIPVL_ERR_INVALID_ARG, "zipvl_decode: NULL pointer");
     if ((k_new == NULL) != (v_new == NULL))

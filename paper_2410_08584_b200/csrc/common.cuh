@@ -159,8 +159,8 @@ size_t decode_partial_bytes(int B, int Hq, int D, int max_len);
 zipvl_status launch_decode_merge(int dtype, int D, int Hq, int B, int chunk, int n_chunks, const float *ws,
                                  const int *lens, int32_t *seq_lens, void *out, cudaStream_t st,
                                  const int *used = nullptr, int group = 1);
-// Grouped-query decode on the tensor cores: 16-bit storage, head_dim 128, 2 to 32 query heads per
-// kv head.  Two kernels that leave partials in the layout of the kernels in decode.cu and the
+// Grouped-query decode on the tensor cores: 16-bit storage, head_dim 64 / 96 / 128, 2 to 32 query
+// heads per kv head.  Two kernels that leave partials in the layout of the kernels in decode.cu and the
 // (length, appended) pairs in lens[]; the caller launches the merge.
 //   decode_tc.cu             one CTA per chunk of a (request, kv head): one partial per chunk, returns
 //                            the chunk it used (never smaller than min_chunk);

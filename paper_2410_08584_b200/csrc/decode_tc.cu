@@ -1,6 +1,6 @@
 // Grouped-query decode over the kept cache on the 5th-generation tensor cores
 // (Algorithm 2; Eq. 4 append, Eq. 5 attention of one query token over the whole cache).
-// 16-bit storage, head_dim 128, 2 to 32 query heads per key/value head.
+// 16-bit storage, head_dim 64, 96 or 128, 2 to 32 query heads per key/value head.
 //
 // With G query heads sharing one cached row, the CUDA-core kernel needs 2*G multiply-adds per
 // cached element; from G = 4 on that, not HBM, sets its pace.  Here the G query rows of a
@@ -88,7 +88,9 @@ struct DtMerge {
 constexpr size_t kDtSmem = kTileBytes * (1 + kSlots) + sizeof(DtBarriers) + 1024;
 static_assert(sizeof(DtMerge) <= kTileBytes * kSlots, "the merge staging reuses the ring");
 
-template <bool kHalf, bool kPaged>
+// HD: head_dim (64, 96 or 128); the shared-memory tiles stay 128 wide and the narrower heads use
+// the front of them
+template <bool kHalf, bool kPaged, int HD>
 __global__ void __launch_bounds__(kThreadsDt, 1)
 decode_tc_kernel(int Hq, int Hkv, float scale_log2, const __nv_bfloat16 *__restrict__ q,
                  const __nv_bfloat16 *__restrict__ k_new, const __nv_bfloat16 *__restrict__ v_new,
@@ -141,7 +143,7 @@ decode_tc_kernel(int Hq, int Hkv, float scale_log2, const __nv_bfloat16 *__restr
     if (c0 >= len) {
         // a chunk past the request's length: empty partials (the merge reads every chunk slot)
         if ((int)threadIdx.x < G) {
-            float *dst = ws + (((long long)b * Hq + h0 + threadIdx.x) * n_chunks + blockIdx.x) * (kD + 2);
+            float *dst = ws + (((long long)b * Hq + h0 + threadIdx.x) * n_chunks + blockIdx.x) * (HD + 2);
             dst[0] = -INFINITY;
             dst[1] = 0.f;
         }
@@ -170,7 +172,7 @@ decode_tc_kernel(int Hq, int Hkv, float scale_log2, const __nv_bfloat16 *__restr
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = bar->tmem_base;
-    const long long row_pitch = (long long)Hkv * kD;          // elements between cache rows
+    const long long row_pitch = (long long)Hkv * HD;          // elements between cache rows
 
     if (warp >= 4 && warp < kIssuerWarp) {
         // ------------------------------ producers ------------------------------
@@ -178,9 +180,9 @@ decode_tc_kernel(int Hq, int Hkv, float scale_log2, const __nv_bfloat16 *__restr
         const int group = (warp - 4) >> 2;
         const int c = lane & 15, sub = lane >> 4;
         const int32_t *my_table = kPaged ? pg.table + (long long)b * pg.stride : nullptr;
-        const __nv_bfloat16 *new_k = k_new ? k_new + ((long long)b * Hkv + g) * kD : nullptr;
-        const __nv_bfloat16 *new_v = v_new ? v_new + ((long long)b * Hkv + g) * kD : nullptr;
-        const long long head_off = coff + (long long)g * kD;
+        const __nv_bfloat16 *new_k = k_new ? k_new + ((long long)b * Hkv + g) * HD : nullptr;
+        const __nv_bfloat16 *new_v = v_new ? v_new + ((long long)b * Hkv + g) * HD : nullptr;
+        const long long head_off = coff + (long long)g * HD;
         long long my_off = -1;                  // cache offset (elements) of row 32p + lane of the tile
         const int total = 2 * n_tiles;          // K0 V0 K1 V1 ...
         // this group's share of the sequence: seq = group + j * kGroups
@@ -214,14 +216,16 @@ decode_tc_kernel(int Hq, int Hkv, float scale_log2, const __nv_bfloat16 *__restr
                 const long long off = __shfl_sync(0xffffffffu, my_off, i + 16 * sub);
                 const uint32_t dst = tile + r * 128 + (c >> 3) * kHalfBytes + (((c & 7) ^ (r & 7)) << 4);
                 const bool ok = off >= 0;
-                const __nv_bfloat16 *src = cache + (ok ? off : 0) + head_off + c * 8;
+                const bool piece = c < HD / 8;                          // (a row has HD / 8 chunks of 16 bytes)
+                const __nv_bfloat16 *src = cache + (ok ? off : 0) + head_off + (piece ? c : 0) * 8;
                 if (ok && j0 + r == new_row) {
                     // the appended token: read from k_new / v_new, stored into the cache on the way
-                    src = fresh + c * 8;
-                    *reinterpret_cast<uint4 *>(cache + off + head_off + c * 8) =
-                        *reinterpret_cast<const uint4 *>(src);
+                    src = fresh + (piece ? c : 0) * 8;
+                    if (piece)
+                        *reinterpret_cast<uint4 *>(cache + off + head_off + c * 8) =
+                            *reinterpret_cast<const uint4 *>(src);
                 }
-                cp_async16(dst, src, ok ? 16u : 0u);
+                cp_async16(dst, src, (ok && piece) ? 16u : 0u);
             }
             cp_async_commit();
         };
@@ -252,7 +256,7 @@ decode_tc_kernel(int Hq, int Hkv, float scale_log2, const __nv_bfloat16 *__restr
         // ------------------------------ MMA issuer ------------------------------
         const bool leader = elect_one();
         constexpr uint32_t idesc_qk = idesc_f16kind(128, kBN, false, false, !kHalf);
-        constexpr uint32_t idesc_pv = idesc_f16kind(128, kD, false, true, !kHalf);
+        constexpr uint32_t idesc_pv = idesc_f16kind(128, HD, false, true, !kHalf);
         constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
         const uint32_t lo_q = ((sQ & 0x3FFFFu) >> 4) | (1u << 16);
         const uint32_t lo_ring = (sRing & 0x3FFFFu) >> 4;
@@ -269,7 +273,7 @@ decode_tc_kernel(int Hq, int Hkv, float scale_log2, const __nv_bfloat16 *__restr
             const uint32_t d = tmem + kColS + (n & 1) * 128;
             if (leader && !*abort_flag) {
 #pragma unroll
-                for (int kb = 0; kb < kD / 16; ++kb) {
+                for (int kb = 0; kb < HD / 16; ++kb) {
                     const uint32_t o = ((kb >> 2) * kHalfBytes + (kb & 3) * 32) >> 4;
                     mma_ss(d, desc(lo_q + o), desc(lo_k + o), idesc_qk, kb > 0);
                 }
@@ -320,7 +324,7 @@ decode_tc_kernel(int Hq, int Hkv, float scale_log2, const __nv_bfloat16 *__restr
                 if (r < G) {
                     const int row = w * 32 + r;
                     cp_async16(sQ + row * 128 + (c >> 3) * kHalfBytes + (((c & 7) ^ (row & 7)) << 4),
-                               q + ((long long)b * Hq + h0 + r) * kD + c * 8, 16u);
+                               q + ((long long)b * Hq + h0 + r) * HD + c * 8, c < HD / 8 ? 16u : 0u);
                 }
             }
             cp_async_commit();
@@ -368,7 +372,7 @@ decode_tc_kernel(int Hq, int Hkv, float scale_log2, const __nv_bfloat16 *__restr
                 mbar_wait(smem_u32(&bar->pv_done), (n - 1) & 1, abort_flag);
                 tc_fence_after();
 #pragma unroll 1
-                for (int cc = 0; cc < 4; ++cc) {
+                for (int cc = 0; cc < HD / 32; ++cc) {
                     uint32_t r[32];
                     tmem_ld32(tO + cc * 32, r);
                     tmem_wait_ld();
@@ -405,7 +409,7 @@ decode_tc_kernel(int Hq, int Hkv, float scale_log2, const __nv_bfloat16 *__restr
             mg->l[w][lane] = l;
         }
 #pragma unroll 1
-        for (int cc = 0; cc < 4; ++cc) {
+        for (int cc = 0; cc < HD / 32; ++cc) {
             uint32_t r[32];
             tmem_ld32(tO + cc * 32, r);
             tmem_wait_ld();
@@ -428,11 +432,11 @@ decode_tc_kernel(int Hq, int Hkv, float scale_log2, const __nv_bfloat16 *__restr
                 if (mr != -INFINITY) {
                     const float wgt = ex2(mr - M);
                     Ls += mg->l[x][hh] * wgt;
-                    Os += mg->o[x][hh][ch] * wgt;
+                    Os += mg->o[x][hh][ch < HD ? ch : 0] * wgt;
                 }
             }
-            float *dst = ws + (((long long)b * Hq + h0 + hh) * n_chunks + blockIdx.x) * (kD + 2);
-            dst[2 + ch] = Os;
+            float *dst = ws + (((long long)b * Hq + h0 + hh) * n_chunks + blockIdx.x) * (HD + 2);
+            if (ch < HD) dst[2 + ch] = Os;
             if (ch == 0) { dst[0] = M; dst[1] = Ls; }
         }
     }
@@ -451,7 +455,7 @@ decode_tc_kernel(int Hq, int Hkv, float scale_log2, const __nv_bfloat16 *__restr
 bool decode_tc_supported(const zipvl_decode_desc &d) {
     if (d.n_kv_heads < 1 || d.n_q_heads % d.n_kv_heads) return false;
     const int G = d.n_q_heads / d.n_kv_heads;
-    return (d.dtype == ZIPVL_BF16 || d.dtype == ZIPVL_F16) && d.head_dim == kD && G >= 2 && G <= kMaxGroup;
+    return (d.dtype == ZIPVL_BF16 || d.dtype == ZIPVL_F16) && (d.head_dim == 128 || d.head_dim == 96 || d.head_dim == 64) && G >= 2 && G <= kMaxGroup;
 }
 
 zipvl_status launch_decode_tc(const zipvl_decode_desc &d, float scale_log2, const void *q,
@@ -473,7 +477,9 @@ zipvl_status launch_decode_tc(const zipvl_decode_desc &d, float scale_log2, cons
     cudaError_t e = cudaSuccess;
 #define ZIPVL_DT(H_, P_)                                                                            \
     {                                                                                               \
-        auto kernel = decode_tc_kernel<H_, P_>;                                                     \
+        auto kernel = decode_tc_kernel<H_, P_, 128>;                                                \
+        if (d.head_dim == 96) kernel = decode_tc_kernel<H_, P_, 96>;                                \
+        if (d.head_dim == 64) kernel = decode_tc_kernel<H_, P_, 64>;                                                     \
         e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDtSmem); \
         if (e == cudaSuccess)                                                                       \
             e = launch_dependent(kernel, dim3(n_chunks, Hkv, B), dim3(kThreadsDt), kDtSmem, st, Hq, Hkv, \

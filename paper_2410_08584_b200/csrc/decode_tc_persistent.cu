@@ -1,7 +1,7 @@
 // Grouped-query decode over the kept cache on the 5th-generation tensor cores: the persistent
 // kernel for large batches (decode_tc.cu holds the one for small ones).
 // (Algorithm 2; Eq. 4 append, Eq. 5 attention of one query token over the whole cache).
-// 16-bit storage, head_dim 128, 2 to 32 query heads per key/value head.
+// 16-bit storage, head_dim 64, 96 or 128, 2 to 32 query heads per key/value head.
 //
 // With G query heads sharing one cached row, the CUDA-core kernel needs 2*G multiply-adds per
 // cached element; from G = 3 on that, not HBM, sets its pace.  Here the G query rows of a kv head
@@ -171,7 +171,9 @@ struct Walker {
     }
 };
 
-template <bool kHalf, bool kPaged>
+// HD: head_dim (64, 96 or 128); the shared-memory tiles stay 128 wide and the narrower heads use
+// the front of them
+template <bool kHalf, bool kPaged, int HD>
 __global__ void __launch_bounds__(kBoundThreadsDt, 1)
 decode_tcp_kernel(DtArgs a) {
     extern __shared__ unsigned char smem_raw[];
@@ -259,7 +261,7 @@ decode_tcp_kernel(DtArgs a) {
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = bar->tmem_base;
-    const long long row_pitch = (long long)a.Hkv * kD;          // elements between cache rows
+    const long long row_pitch = (long long)a.Hkv * HD;          // elements between cache rows
     Walker<kPaged> wk;
     wk.start(a, bar->start_b, bar->start_R, lo);
 
@@ -280,7 +282,7 @@ decode_tcp_kernel(DtArgs a) {
             at = n;
             const int j0 = wk.t * kBN;                   // first cache row of the tile
             const int32_t *my_table = kPaged ? a.pg.table + (long long)wk.b * a.pg.stride : nullptr;
-            const long long head_off = wk.r.coff + (long long)wk.g * kD;
+            const long long head_off = wk.r.coff + (long long)wk.g * HD;
             // one lane per row: where the row lives (-1: behind the length, or in a page outside
             // the pool, which is reported and left out of the attention)
             long long my_off = -1;
@@ -301,21 +303,23 @@ decode_tcp_kernel(DtArgs a) {
             const uint32_t tile = sRing + (seq % kSlots) * kTileBytes;
             __nv_bfloat16 *cache = kind ? a.v_cache : a.k_cache;
             const __nv_bfloat16 *fresh = (kind ? a.v_new : a.k_new);
-            if (fresh) fresh += ((long long)wk.b * a.Hkv + wk.g) * kD;
+            if (fresh) fresh += ((long long)wk.b * a.Hkv + wk.g) * HD;
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
                 const int r = p * 32 + i + 16 * sub;                    // row of the tile
                 const long long off = __shfl_sync(0xffffffffu, my_off, i + 16 * sub);
                 const uint32_t dst = tile + r * 128 + (c >> 3) * kHalfBytes + (((c & 7) ^ (r & 7)) << 4);
                 const bool ok = off >= 0;
-                const __nv_bfloat16 *src = cache + (ok ? off : 0) + head_off + c * 8;
+                const bool piece = c < HD / 8;                          // (a row has HD / 8 chunks of 16 bytes)
+                const __nv_bfloat16 *src = cache + (ok ? off : 0) + head_off + (piece ? c : 0) * 8;
                 if (ok && j0 + r == wk.r.new_row) {
                     // the appended token: read from k_new / v_new, stored into the cache on the way
-                    src = fresh + c * 8;
-                    *reinterpret_cast<uint4 *>(cache + off + head_off + c * 8) =
-                        *reinterpret_cast<const uint4 *>(src);
+                    src = fresh + (piece ? c : 0) * 8;
+                    if (piece)
+                        *reinterpret_cast<uint4 *>(cache + off + head_off + c * 8) =
+                            *reinterpret_cast<const uint4 *>(src);
                 }
-                cp_async16(dst, src, ok ? 16u : 0u);
+                cp_async16(dst, src, (ok && piece) ? 16u : 0u);
             }
             cp_async_commit();
         };
@@ -347,7 +351,7 @@ decode_tcp_kernel(DtArgs a) {
         if (warp == kIssuerWarp) {
         const bool leader = elect_one();
         constexpr uint32_t idesc_qk = idesc_f16kind(128, kBN, false, false, !kHalf);
-        constexpr uint32_t idesc_pv = idesc_f16kind(128, kD, false, true, !kHalf);
+        constexpr uint32_t idesc_pv = idesc_f16kind(128, HD, false, true, !kHalf);
         constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
         const uint32_t lo_q = ((sQ & 0x3FFFFu) >> 4) | (1u << 16);
         const uint32_t lo_ring = (sRing & 0x3FFFFu) >> 4;
@@ -377,7 +381,7 @@ decode_tcp_kernel(DtArgs a) {
             const uint32_t d = tmem + kColS + (n & 1) * 128;
             if (leader && !*abort_flag) {
 #pragma unroll
-                for (int kb = 0; kb < kD / 16; ++kb) {
+                for (int kb = 0; kb < HD / 16; ++kb) {
                     const uint32_t o = ((kb >> 2) * kHalfBytes + (kb & 3) * 32) >> 4;
                     mma_ss(d, desc(lo_q + o), desc(lo_k + o), idesc_qk, kb > 0);
                 }
@@ -434,7 +438,7 @@ decode_tcp_kernel(DtArgs a) {
                 if (r < G) {
                     const int row = w * 32 + o + r;
                     cp_async16(sQ + row * 128 + (c >> 3) * kHalfBytes + (((c & 7) ^ (row & 7)) << 4),
-                               a.q + ((long long)b * a.Hq + g * G + r) * kD + c * 8, 16u);
+                               a.q + ((long long)b * a.Hq + g * G + r) * HD + c * 8, c < HD / 8 ? 16u : 0u);
                 }
             }
             cp_async_commit();
@@ -498,7 +502,7 @@ decode_tcp_kernel(DtArgs a) {
                     mbar_wait(smem_u32(&bar->pv_done), (nn - 1) & 1, abort_flag);
                     tc_fence_after();
 #pragma unroll 1
-                    for (int cc = 0; cc < 4; ++cc) {
+                    for (int cc = 0; cc < HD / 32; ++cc) {
                         uint32_t r[32];
                         tmem_ld32(tO + cc * 32, r);
                         tmem_wait_ld();
@@ -529,13 +533,13 @@ decode_tcp_kernel(DtArgs a) {
             const long long pair0 = wk.pair_start(a);
             const int first_cta = (int)(pair0 / q);
             const int slot = kSoftmaxWarps * ((int)blockIdx.x - first_cta) + w;
-            float *dst = a.ws + (((long long)wk.b * a.Hq + wk.g * G + (lane - off)) * a.n_slots + slot) * (kD + 2);
+            float *dst = a.ws + (((long long)wk.b * a.Hq + wk.g * G + (lane - off)) * a.n_slots + slot) * (HD + 2);
             if (mine) {
                 dst[0] = m;
                 dst[1] = l;
             }
 #pragma unroll 1
-            for (int cc = 0; cc < 4; ++cc) {
+            for (int cc = 0; cc < HD / 32; ++cc) {
                 uint32_t r[32];
                 tmem_ld32(tO + cc * 32, r);
                 tmem_wait_ld();
@@ -569,7 +573,7 @@ decode_tcp_kernel(DtArgs a) {
 bool decode_tcp_supported(const zipvl_decode_desc &d) {
     if (d.n_kv_heads < 1 || d.n_q_heads % d.n_kv_heads) return false;
     const int G = d.n_q_heads / d.n_kv_heads;
-    return (d.dtype == ZIPVL_BF16 || d.dtype == ZIPVL_F16) && d.head_dim == kD && G >= 2 && G <= kMaxGroup;
+    return (d.dtype == ZIPVL_BF16 || d.dtype == ZIPVL_F16) && (d.head_dim == 128 || d.head_dim == 96 || d.head_dim == 64) && G >= 2 && G <= kMaxGroup;
 }
 
 zipvl_status launch_decode_tcp(const zipvl_decode_desc &d, float scale_log2, const void *q,
@@ -601,7 +605,9 @@ zipvl_status launch_decode_tcp(const zipvl_decode_desc &d, float scale_log2, con
     cudaError_t e = cudaSuccess;
 #define ZIPVL_DT(H_, P_)                                                                            \
     {                                                                                               \
-        auto kernel = decode_tcp_kernel<H_, P_>;                                                     \
+        auto kernel = decode_tcp_kernel<H_, P_, 128>;                                               \
+        if (d.head_dim == 96) kernel = decode_tcp_kernel<H_, P_, 96>;                               \
+        if (d.head_dim == 64) kernel = decode_tcp_kernel<H_, P_, 64>;                                                     \
         e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDtSmem); \
         if (e == cudaSuccess)                                                                       \
             e = launch_dependent(kernel, dim3(grid), dim3(kThreadsDt), kDtSmem, st, a);             \

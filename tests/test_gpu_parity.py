@@ -725,6 +725,7 @@ def build_caches(lens, Hkv, d, dtype, extra, seed):
     ([300, 7], 4, 4, 64, torch.float32),
     ([129], 6, 2, 128, torch.float32),
     ([400, 130, 1], 6, 2, 96, torch.bfloat16),
+    ([900, 259, 3], 14, 2, 64, torch.bfloat16),
     ([257, 90], 4, 4, 96, torch.float16),
     ([300, 7], 4, 2, 96, torch.float32),
     # grouped-query heads on the tensor cores: 2, 7, 16 and 32 query heads per kv head, an empty
@@ -771,16 +772,18 @@ def test_decode_parity(zipvl, lens, Hq, Hkv, d, dtype):
     assert st.item() & zipvl.DEV_CAPACITY and np.array_equal(seq_d.cpu().numpy(), seq_o)
 
 
-@pytest.mark.parametrize("lens,Hq,Hkv,dtype", [
-    ([513, 40, 2000], 14, 2, torch.bfloat16),
-    ([5000, 129, 0, 3000, 1], 28, 4, torch.bfloat16),
-    ([2100, 640], 32, 2, torch.float16),
+@pytest.mark.parametrize("lens,Hq,Hkv,d,dtype", [
+    ([513, 40, 2000], 14, 2, 128, torch.bfloat16),
+    ([5000, 129, 0, 3000, 1], 28, 4, 128, torch.bfloat16),
+    ([2100, 640], 32, 2, 128, torch.float16),
+    ([900, 259, 3], 14, 2, 64, torch.bfloat16),          # narrower heads: the front of the 128-wide tiles
+    ([400, 1300], 12, 4, 96, torch.float16),
 ])
-def test_decode_parity_on_the_persistent_kernel(zipvl, monkeypatch, lens, Hq, Hkv, dtype):
+def test_decode_parity_on_the_persistent_kernel(zipvl, monkeypatch, lens, Hq, Hkv, d, dtype):
     """The decode parity test (three steps with appends, a step without, a full cache) with the
     persistent tensor-core kernel forced: by default it only takes large batches."""
     monkeypatch.setenv("ZIPVL_DECODE_KERNEL", "tcp")
-    test_decode_parity(zipvl, lens, Hq, Hkv, 128, dtype)
+    test_decode_parity(zipvl, lens, Hq, Hkv, d, dtype)
 
 
 @pytest.mark.parametrize("lens,Hq,Hkv,dtype,page_rows", [
