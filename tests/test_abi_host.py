@@ -107,8 +107,11 @@ def test_argument_validation_without_a_device(lib):
     assert lib.zipvl_decode(C.byref(d), p, p, null, p, p, p, p, p, 10, p, p, 1 << 20, None, None) == 1
     assert lib.zipvl_decode(C.byref(d), p, p, p, p, p, p, p, p, 0, p, p, 1 << 20, None, None) == 1
     assert lib.zipvl_decode(C.byref(d), p, p, p, p, p, p, p, p, 10, p, p, 8, None, None) == 3
-    d9 = z.zipvl_decode_desc(2, 18, 2, 64, 0, 0.0)
+    # query heads per kv head: beyond 8 in fp32, beyond 32 in 16-bit storage
+    d9 = z.zipvl_decode_desc(2, 18, 2, 64, z.ZIPVL_F32, 0.0)
     assert lib.zipvl_decode(C.byref(d9), p, p, p, p, p, p, p, p, 10, p, p, 1 << 20, None, None) == 2
+    d33 = z.zipvl_decode_desc(2, 66, 2, 64, z.ZIPVL_BF16, 0.0)
+    assert lib.zipvl_decode(C.byref(d33), p, p, p, p, p, p, p, p, 10, p, p, 1 << 20, None, None) == 2
     # decode without a workspace: the same validation, and the size check of its built-in
     # scratch, before anything is launched
     na = lib.zipvl_decode_noalloc
