@@ -69,7 +69,7 @@ constexpr int kThreadsDt = 32 * (kIssuerWarp + 1);
 constexpr int kBoundThreadsDt = 640;
 constexpr uint32_t kTmemColsDt = 512;
 constexpr uint32_t kColS = 0, kColP = 256, kColO = 384;
-constexpr int kMaxGroup = 32;
+constexpr int kMaxGroup = 32;       // query heads per kv head: one warp's 32 rows of the tile
 constexpr float kRescaleBf16 = 32.0f, kRescaleHalf = 8.0f;   // octaves the running max may lag
 
 struct DtBarriers {
@@ -570,17 +570,13 @@ decode_tcp_kernel(DtArgs a) {
 
 }  // namespace
 
-bool decode_tcp_supported(const zipvl_decode_desc &d) {
-    if (d.n_kv_heads < 1 || d.n_q_heads % d.n_kv_heads) return false;
-    const int G = d.n_q_heads / d.n_kv_heads;
-    return (d.dtype == ZIPVL_BF16 || d.dtype == ZIPVL_F16) && (d.head_dim == 128 || d.head_dim == 96 || d.head_dim == 64) && G >= 2 && G <= kMaxGroup;
-}
-
 zipvl_status launch_decode_tcp(const zipvl_decode_desc &d, float scale_log2, const void *q,
                               const void *k_new, const void *v_new, void *k_cache, void *v_cache,
                               const int64_t *cache_off, PageArgs pg, const int32_t *capacity,
                               int32_t *seq_lens, int max_len, int n_slots, float *partials, int *lens,
                               int *used, int32_t *status_word, cudaStream_t st) {
+    if (!decode_tc_supported(d) || d.n_q_heads / d.n_kv_heads > kMaxGroup)
+        return fail(ZIPVL_ERR_UNSUPPORTED, "zipvl_decode: this shape does not run on the tensor-core kernel");
     static int n_sm_of[64] = {0};                  // multiprocessors per device, asked once
     int dev = 0;
     cudaGetDevice(&dev);
@@ -607,7 +603,7 @@ zipvl_status launch_decode_tcp(const zipvl_decode_desc &d, float scale_log2, con
     {                                                                                               \
         auto kernel = decode_tcp_kernel<H_, P_, 128>;                                               \
         if (d.head_dim == 96) kernel = decode_tcp_kernel<H_, P_, 96>;                               \
-        if (d.head_dim == 64) kernel = decode_tcp_kernel<H_, P_, 64>;                                                     \
+        if (d.head_dim == 64) kernel = decode_tcp_kernel<H_, P_, 64>;                               \
         e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDtSmem); \
         if (e == cudaSuccess)                                                                       \
             e = launch_dependent(kernel, dim3(grid), dim3(kThreadsDt), kDtSmem, st, a);             \

@@ -831,6 +831,41 @@ def test_decode_kernel_choice_can_be_forced_and_both_match_the_oracle(zipvl, mon
         check_attention(to_np(a), to_np(b).astype(np.float64), dtype)
 
 
+@pytest.mark.parametrize("kernel,B,Hq,Hkv", [
+    ("tcp", 700, 8, 2),        # more requests than the CTA has threads: the length scan takes several each
+    ("tcp", 1500, 12, 4),      # far more (request, kv head) pairs than CTAs: dozens of segments per CTA
+    ("tc", 700, 8, 2),
+    ("simt", 700, 8, 8),
+])
+def test_decode_on_many_short_requests(zipvl, monkeypatch, kernel, B, Hq, Hkv):
+    """Hundreds of requests of zero to a few hundred rows, a few long ones among them, one step with
+    an appended token: every request's output, length and appended row against the oracle."""
+    monkeypatch.setenv("ZIPVL_DECODE_KERNEL", kernel)
+    d, dtype = 128, torch.bfloat16
+    rng = np.random.default_rng(B + Hq)
+    lens = [int(x) for x in rng.integers(0, 400, size=B)]
+    for b in rng.choice(B, size=5, replace=False):
+        lens[int(b)] = int(rng.integers(2000, 5000))
+    lens[3], lens[B - 1] = 0, 1
+    kc, vc, off, cap = build_caches(lens, Hkv, d, dtype, 1, seed=B)
+    g = torch.Generator().manual_seed(B)
+    q = torch.randn(B, Hq, d, generator=g).to(dtype)
+    kn = torch.randn(B, Hkv, d, generator=g).to(dtype)
+    vn = torch.randn(B, Hkv, d, generator=g).to(dtype)
+    desc = zipvl.zipvl_decode_desc(B, Hq, Hkv, d, zipvl.ZIPVL_BF16, 0.0)
+    kc_d, vc_d, off_d, cap_d = kc.to(DEV), vc.to(DEV), off.to(DEV), cap.to(DEV)
+    seq_d = torch.tensor(lens, dtype=torch.int32, device=DEV)
+    st = status_word()
+    out = zipvl.zipvl_decode(desc, q.to(DEV), kn.to(DEV), vn.to(DEV), kc_d, vc_d, off_d, cap_d, seq_d,
+                             max(lens) + 1, status=st)
+    ko, vo, seqo = kc.float().numpy().copy(), vc.float().numpy().copy(), np.array(lens, np.int32)
+    ref = oracle.decode_step(to_np(q), to_np(kn), to_np(vn), ko, vo, off.numpy(), seqo, Hkv)
+    assert st.item() == 0
+    check_attention(to_np(out), ref, dtype)
+    assert np.array_equal(seq_d.cpu().numpy(), seqo) and np.array_equal(seqo, np.array(lens) + 1)
+    assert np.array_equal(kc_d.float().cpu().numpy(), ko) and np.array_equal(vc_d.float().cpu().numpy(), vo)
+
+
 @pytest.mark.parametrize("lens,Hq,Hkv,d,dtype,page_rows", [
     ([700, 1, 300, 1025, 17, 0], 8, 8, 128, torch.bfloat16, 64),
     ([513, 40, 2000], 14, 2, 128, torch.bfloat16, 128),
