@@ -269,68 +269,88 @@ decode_kernel(int Hq, int Hkv, float scale_log2, const T *__restrict__ q,
 // Second kernel of a step: merges the per-chunk partial results of one request's query
 // heads (online-softmax merge), writes the output, and bumps the request's length.
 // Launched as a programmatic dependent of the kernel above, so it is staged while that one
-// runs; no tickets, no counters to clear.  Eight adjacent lanes share one (head, channel):
-// lane p takes chunks p, p + 8, ... -- every chunk slot holds a partial, an empty one past the
-// request's length, so all loads go out at once without waiting for the length -- and the
-// eight are merged by shuffles in a fixed order.
-constexpr int kMergeLanes = 8;
+// runs; no tickets, no counters to clear.  `lanes` (1, 2, 4 or 8) adjacent lanes share two
+// channels of one head: lane p takes chunks p, p + lanes, ... -- every chunk slot holds a
+// partial, an empty one past the request's length, so all loads go out at once without waiting
+// for the length -- and the lanes are merged by shuffles in a fixed order.  The host picks
+// `lanes` so that a batch of many requests does not become thousands of CTAs with one load
+// each (merge_lanes below).
+__device__ __forceinline__ void store2(float *p, float a, float b) { *reinterpret_cast<float2 *>(p) = make_float2(a, b); }
+__device__ __forceinline__ void store2(__nv_bfloat16 *p, float a, float b) {
+    *reinterpret_cast<__nv_bfloat162 *>(p) = __floats2bfloat162_rn(a, b);
+}
+__device__ __forceinline__ void store2(__half *p, float a, float b) { *reinterpret_cast<__half2 *>(p) = __floats2half2_rn(a, b); }
+
 template <typename T, int D>
 __global__ void __launch_bounds__(256)
-decode_merge_kernel(int Hq, int chunk, int n_chunks, const float *__restrict__ ws,
+decode_merge_kernel(int Hq, int lanes, int n_chunks, const float *__restrict__ ws,
                     const int *__restrict__ lens, int32_t *__restrict__ seq_lens, T *__restrict__ out,
                     const int *__restrict__ used, int group) {
+    static_assert(D % 2 == 0, "two channels per thread");
     grid_launch_dependents();
     grid_dependency_wait(ws, lens, seq_lens, used);
     const int b = blockIdx.y;
-    const int t = (blockIdx.x * 256 + threadIdx.x) / kMergeLanes;       // (head, channel) of this lane group
-    const int part = threadIdx.x % kMergeLanes;
-    const bool live = t < Hq * D;
-    const int hq = live ? t / D : 0, c = live ? t % D : 0;
+    const int t = (blockIdx.x * 256 + threadIdx.x) / lanes;             // (head, channel pair) of this lane group
+    const int part = threadIdx.x % lanes;
+    const bool live = t < Hq * (D / 2);
+    const int hq = live ? t / (D / 2) : 0, c = live ? 2 * (t % (D / 2)) : 0;
     const float *src = ws + ((long long)b * Hq + hq) * n_chunks * (D + 2);
     // the tensor-core kernel fills only the first used[request, kv head] slots of a head
     const int n_used = used ? min(n_chunks, max(0, used[b * (Hq / group) + hq / group])) : n_chunks;
-    float M = -INFINITY, Ls = 0.f, Os = 0.f;
-    for (int i0 = part; i0 < n_used; i0 += 8 * kMergeLanes) {
-        float mi[8], li[8], oi[8];
+    float M = -INFINITY, Ls = 0.f, O0 = 0.f, O1 = 0.f;
+    for (int i0 = part; i0 < n_used; i0 += 8 * lanes) {
+        float2 ml[8], oi[8];
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
-            const int i = i0 + u * kMergeLanes;
+            const int i = i0 + u * lanes;
             const bool in = live && i < n_used;
-            const float *p = src + (long long)(in ? i : 0) * (D + 2);
-            mi[u] = in ? __ldcg(p) : -INFINITY;
-            li[u] = in ? __ldcg(p + 1) : 0.f;
-            oi[u] = in ? __ldcg(p + 2 + c) : 0.f;
+            const float *p = src + (long long)(in ? i : 0) * (D + 2);   // (a slot is (D + 2) * 4 bytes: 8-byte aligned)
+            ml[u] = in ? __ldcg(reinterpret_cast<const float2 *>(p)) : make_float2(-INFINITY, 0.f);
+            oi[u] = in ? __ldcg(reinterpret_cast<const float2 *>(p + 2 + c)) : make_float2(0.f, 0.f);
         }
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
-            if (mi[u] != -INFINITY) {
-                const float Mn = fmaxf(M, mi[u]);
-                const float wo = fast_exp2(M - Mn), wn = fast_exp2(mi[u] - Mn);
-                Ls = Ls * wo + li[u] * wn;
-                Os = Os * wo + oi[u] * wn;
+            if (ml[u].x != -INFINITY) {
+                const float Mn = fmaxf(M, ml[u].x);
+                const float wo = fast_exp2(M - Mn), wn = fast_exp2(ml[u].x - Mn);
+                Ls = Ls * wo + ml[u].y * wn;
+                O0 = O0 * wo + oi[u].x * wn;
+                O1 = O1 * wo + oi[u].y * wn;
                 M = Mn;
             }
         }
     }
-#pragma unroll
-    for (int o = 1; o < kMergeLanes; o <<= 1) {
+    for (int o = 1; o < lanes; o <<= 1) {
         const float M2 = __shfl_xor_sync(0xffffffffu, M, o);
         const float L2 = __shfl_xor_sync(0xffffffffu, Ls, o);
-        const float O2 = __shfl_xor_sync(0xffffffffu, Os, o);
+        const float P0 = __shfl_xor_sync(0xffffffffu, O0, o);
+        const float P1 = __shfl_xor_sync(0xffffffffu, O1, o);
         const float Mn = fmaxf(M, M2);
         // (the two sides of a pair compute the same sum in the same order of operands)
         const float w1 = (M == -INFINITY) ? 0.f : fast_exp2(M - Mn);
         const float w2 = (M2 == -INFINITY) ? 0.f : fast_exp2(M2 - Mn);
         const bool lo = (part & o) == 0;
         Ls = lo ? (Ls * w1 + L2 * w2) : (L2 * w2 + Ls * w1);
-        Os = lo ? (Os * w1 + O2 * w2) : (O2 * w2 + Os * w1);
+        O0 = lo ? (O0 * w1 + P0 * w2) : (P0 * w2 + O0 * w1);
+        O1 = lo ? (O1 * w1 + P1 * w2) : (P1 * w2 + O1 * w1);
         M = Mn;
     }
     // (an empty cache with nothing appended has only empty partials: the output is zero)
-    if (live && part == 0) store_elem(out + ((long long)b * Hq + hq) * D + c, Ls > 0.f ? Os / Ls : 0.f);
+    if (live && part == 0)
+        store2(out + ((long long)b * Hq + hq) * D + c, Ls > 0.f ? O0 / Ls : 0.f, Ls > 0.f ? O1 / Ls : 0.f);
     // Eq. 4: the appended row now counts
     if (blockIdx.x == 0 && threadIdx.x == 0 && lens[2 * b + 1]) seq_lens[b] = lens[2 * b];
 }
+
+// Lanes per (head, channel pair) of the merge: as many as there are slots to share (at most
+// 8), but no more than keep the whole launch within about one wave of threads -- with hundreds
+// of requests the merge is bound by the number of CTAs it starts, not by its loads.
+int merge_lanes(int B, int Hq, int D, int n_slots) {
+    int lanes = 8;
+    while (lanes > 1 && (lanes / 2 >= n_slots || (long long)B * Hq * (D / 2) * lanes > 148LL * 2048)) lanes >>= 1;
+    return lanes;
+}
+dim3 merge_grid(int B, int Hq, int D, int lanes) { return dim3((Hq * (D / 2) * lanes + 255) / 256, B); }
 
 // Cache rows per CTA: small problems get small chunks so that every SM still has
 // several CTAs in flight (about eight per SM), large ones stream 512 rows per CTA.
@@ -394,10 +414,12 @@ zipvl_status run(const zipvl_decode_desc &d, float scale_log2, const void *q, co
     else ZIPVL_DEC(8)
 #undef ZIPVL_DEC
 #undef ZIPVL_DEC_P
-    if (le == cudaSuccess)
-        le = launch_dependent(decode_merge_kernel<T, D>, dim3((Hq * D * kMergeLanes + 255) / 256, B), dim3(256), 0, st, Hq,
-                              chunk, n_chunks, (const float *)wsf, (const int *)lens, seq_lens, (T *)out,
+    if (le == cudaSuccess) {
+        const int lanes = merge_lanes(B, Hq, D, n_chunks);
+        le = launch_dependent(decode_merge_kernel<T, D>, merge_grid(B, Hq, D, lanes), dim3(256), 0, st, Hq,
+                              lanes, n_chunks, (const float *)wsf, (const int *)lens, seq_lens, (T *)out,
                               (const int *)nullptr, 1);
+    }
     if (le != cudaSuccess) return fail(ZIPVL_ERR_CUDA, "zipvl_decode: launch: %s", cudaGetErrorString(le));
     count_launches(2);
     return check_launch("zipvl_decode");
@@ -413,9 +435,11 @@ zipvl_status launch_decode_merge(int dtype, int D, int Hq, int B, int chunk, int
                                  const int *lens, int32_t *seq_lens, void *out, cudaStream_t st,
                                  const int *used, int group) {
     cudaError_t le = cudaErrorInvalidValue;
-    const dim3 grid((Hq * D * kMergeLanes + 255) / 256, B);
+    (void)chunk;
+    const int lanes = merge_lanes(B, Hq, D, n_chunks);
+    const dim3 grid = merge_grid(B, Hq, D, lanes);
 #define ZIPVL_MERGE(T_, D_) \
-    le = launch_dependent(decode_merge_kernel<T_, D_>, grid, dim3(256), 0, st, Hq, chunk, n_chunks, ws, lens, seq_lens, (T_ *)out, used, group)
+    le = launch_dependent(decode_merge_kernel<T_, D_>, grid, dim3(256), 0, st, Hq, lanes, n_chunks, ws, lens, seq_lens, (T_ *)out, used, group)
     if (dtype == ZIPVL_BF16 && D == 128) ZIPVL_MERGE(__nv_bfloat16, 128);
     else if (dtype == ZIPVL_BF16 && D == 96) ZIPVL_MERGE(__nv_bfloat16, 96);
     else if (dtype == ZIPVL_BF16 && D == 64) ZIPVL_MERGE(__nv_bfloat16, 64);
@@ -438,24 +462,23 @@ zipvl_status dispatch_decode(const zipvl_decode_desc &d, float scale_log2, const
                              const int64_t *cache_off, PageArgs pg, const int32_t *capacity,
                              int32_t *seq_lens, int max_len, void *out, void *ws,
                              int32_t *status_word, cudaStream_t st) {
-    // Grouped-query attention in 16-bit storage at head_dim 128 runs on the tensor cores from
-    // two query heads per kv head on: there the CUDA-core kernel is bound by its multiply-adds
-    // (0.51 of the HBM copy rate at four heads per kv head, 0.27 at seven; at two it still reaches
-    // 0.81).  Of the two tensor-core kernels the persistent one takes the large problems (from
-    // about 14 key/value tiles per SM on it is 5 to 10 % faster: no CTA prologue between work
-    // items); below that the launch of one CTA per chunk is quicker (fewer partials to merge,
-    // shorter CTAs).  ZIPVL_DECODE_KERNEL=simt|tc|tcp overrides the choice (measurements, tests).
+    // Grouped-query attention in 16-bit storage runs on the tensor cores from two query heads per
+    // kv head on: there the CUDA-core kernel is bound by its multiply-adds (0.49 of the HBM copy
+    // rate at four heads per kv head, 0.29 at seven; at two it reaches 0.81 against 0.84).  Of the
+    // two tensor-core kernels the persistent one takes the large problems (from about ten
+    // key/value tiles per SM on it is 5 to 15 % faster: no CTA prologue between work items); below
+    // that the launch of one CTA per chunk is quicker (fewer partials to merge, shorter CTAs).
+    // ZIPVL_DECODE_KERNEL=simt|tc|tcp overrides the choice (measurements, tests).
     {
         const char *env = getenv("ZIPVL_DECODE_KERNEL");
         const int G = d.n_q_heads / d.n_kv_heads;
         const long long tiles = (long long)d.batch * d.n_kv_heads * ((max_len + 127) / 128);
-        // (two query heads per kv head: the CUDA-core kernel is the faster one on large batches,
-        // 0.81 against 0.74 of the copy rate, the chunked tensor-core kernel on small ones)
-        const bool want_simt = env ? !strcmp(env, "simt") : (G < 3 && tiles >= 2000);
+        constexpr long long kPersistentFrom = 1500;
+        const bool want_simt = env && !strcmp(env, "simt");
         if (decode_tc_supported(d) && (!want_simt || G > 8)) {
             const int B = d.batch, Hq = d.n_q_heads, D = d.head_dim;
             const bool persistent = env && !strcmp(env, "tcp") ? true
-                                    : (env && !strcmp(env, "tc") ? false : tiles >= 2000);
+                                    : (env && !strcmp(env, "tc") ? false : tiles >= kPersistentFrom);
             float *wsf = reinterpret_cast<float *>(ws);
             int *lens = reinterpret_cast<int *>(reinterpret_cast<char *>(ws) + partial_bytes(B, Hq, D, max_len, true));
             int *used = lens + 2 * B;
