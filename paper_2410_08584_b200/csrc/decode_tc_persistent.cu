@@ -44,7 +44,7 @@ namespace {
 
 using namespace ptx;
 
-constexpr int kD = 128, kBN = 128;
+constexpr int kBN = 128;
 constexpr int kSlots = 6;              // ring of K / V tiles (K0 V0 K1 V1 K2 V2)
 // A warp can only have so many 16-byte async copies outstanding, so the bytes in flight -- and
 // with them the bandwidth the SM can draw -- grow with the number of producer warps, not with the
@@ -99,7 +99,7 @@ struct DtArgs {
     PageArgs pg;
     const int32_t *capacity;
     int32_t *seq_lens;
-    float *ws;                         // partials: [B][Hq][n_slots][kD + 2]
+    float *ws;                         // partials: [B][Hq][n_slots][head_dim + 2]
     int *lens;                         // (length, appended) per request, for the merge
     int *used;                         // slots in use per (request, kv head), for the merge
     int32_t *status_word;

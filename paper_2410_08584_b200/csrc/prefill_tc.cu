@@ -42,7 +42,7 @@ namespace {
 
 using namespace ptx;
 
-constexpr int kD = 128;               // width of the shared-memory tiles; head_dim 64 and 96 use the front of it
+// (the shared-memory tiles are 128 columns wide; head_dim 64 and 96 use the front of them)
 constexpr int kBM = 128, kBN = 128;   // query / key tile
 constexpr int kPair = 2 * kBM;        // query rows per CTA
 constexpr int kSlots = 5;             // ring of K / V tiles

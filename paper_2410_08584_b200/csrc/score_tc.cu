@@ -27,9 +27,9 @@ namespace {
 
 using namespace ptx;
 
-// kD: the width of the shared-memory tiles (two 64-column swizzle atoms); head_dim 64 and 96 use
-// the front of it -- fewer 16-byte chunks per gathered row, fewer k-blocks per MMA
-constexpr int kD = 128, kTile = 128, kMaxProbe = 128;
+// The shared-memory tiles are 128 columns wide (two 64-column swizzle atoms); head_dim 64 and 96 use
+// the front of them -- fewer 16-byte chunks per gathered row, fewer k-blocks per MMA
+constexpr int kTile = 128, kMaxProbe = 128;
 constexpr int kHalfBytes = 128 * 128;
 constexpr int kTileBytes = 2 * kHalfBytes;
 constexpr int kKStages = 2;

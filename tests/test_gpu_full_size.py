@@ -229,3 +229,81 @@ def test_batched_decode_full_size_compacted_and_dense(zipvl):
         # the appended rows went into the caches bit for bit
         assert np.array_equal(kcache.float().cpu().numpy(), ko) and np.array_equal(vcache.float().cpu().numpy(), vo)
         del kcache, vcache, ko, vo
+
+
+@pytest.mark.parametrize("paged", [False, True])
+def test_grouped_query_decode_full_size(zipvl, paged):
+    """The grouped-query decode configuration bench.py times (16 requests of 6000 to 30000 kept
+    rows, 28 query heads on 4 kv heads, head_dim 128, bf16), on the kernel the library picks at
+    that size: three steps with appended tokens, every output of every request and head, the
+    lengths and the appended rows against the oracle.  Once on contiguous caches, once on a
+    paged pool whose pages are dealt out in a shuffled order."""
+    z = zipvl
+    B, Hq, Hkv, d, steps = 16, 28, 4, 128, 3
+    row = Hkv * d
+    g = torch.Generator().manual_seed(4242)
+    lens = torch.randint(6000, 30001, (B,), generator=g).tolist()
+    caps = [n + steps for n in lens]
+    page_rows = 128
+    if not paged:
+        off = np.concatenate([[0], np.cumsum([c * row for c in caps[:-1]])]).astype(np.int64)
+        total_rows = sum(caps)
+    else:
+        pages_of = [(c + page_rows - 1) // page_rows for c in caps]
+        n_pages = sum(pages_of)
+        perm = torch.randperm(n_pages, generator=g).numpy().astype(np.int32)
+        table = np.full((B, max(pages_of)), -1, np.int32)
+        at = 0
+        for b, n in enumerate(pages_of):
+            table[b, :n] = perm[at: at + n]
+            at += n
+        total_rows = n_pages * page_rows
+    kc = torch.zeros(total_rows * row, dtype=torch.bfloat16)
+    vc = torch.zeros(total_rows * row, dtype=torch.bfloat16)
+
+    def rows_of(b, n):               # element offsets of request b's first n rows
+        if not paged:
+            return off[b] + np.arange(n, dtype=np.int64) * row
+        r = np.arange(n, dtype=np.int64)
+        return (table[b, r // page_rows].astype(np.int64) * page_rows + r % page_rows) * row
+
+    for b, n in enumerate(lens):
+        kv = torch.randn(2, n, row, generator=g).to(torch.bfloat16)
+        at = torch.from_numpy(rows_of(b, n))[:, None] + torch.arange(row)[None, :]
+        kc[at.reshape(-1)] = kv[0].reshape(-1)
+        vc[at.reshape(-1)] = kv[1].reshape(-1)
+    # the oracle works on contiguous per-request caches of its own
+    o_off = np.concatenate([[0], np.cumsum([c * row for c in caps[:-1]])]).astype(np.int64)
+    ko = np.zeros(sum(caps) * row, np.float32)
+    vo = np.zeros(sum(caps) * row, np.float32)
+    for b, n in enumerate(lens):
+        at = (torch.from_numpy(rows_of(b, n))[:, None] + torch.arange(row)[None, :]).reshape(-1)
+        ko[o_off[b]: o_off[b] + n * row] = kc[at].float().numpy()
+        vo[o_off[b]: o_off[b] + n * row] = vc[at].float().numpy()
+    seqo = np.array(lens, np.int32)
+    kc_d, vc_d = kc.to(DEV), vc.to(DEV)
+    seq = torch.tensor(lens, dtype=torch.int32, device=DEV)
+    capt = torch.tensor(caps, dtype=torch.int32, device=DEV)
+    desc = z.zipvl_decode_desc(B, Hq, Hkv, d, z.ZIPVL_BF16, 0.0)
+    st = torch.zeros(1, dtype=torch.int32, device=DEV)
+    for s_ in range(steps):
+        qn = torch.randn(B, Hq, d, generator=g).to(torch.bfloat16)
+        kn = torch.randn(B, Hkv, d, generator=g).to(torch.bfloat16)
+        vn = torch.randn(B, Hkv, d, generator=g).to(torch.bfloat16)
+        if not paged:
+            out = z.zipvl_decode(desc, qn.to(DEV), kn.to(DEV), vn.to(DEV), kc_d, vc_d,
+                                 torch.from_numpy(off).to(DEV), capt, seq, max(caps), status=st)
+        else:
+            out = z.zipvl_decode_paged(desc, qn.to(DEV), kn.to(DEV), vn.to(DEV),
+                                       kc_d.view(n_pages, page_rows, Hkv, d), vc_d.view(n_pages, page_rows, Hkv, d),
+                                       torch.from_numpy(table).to(DEV), capt, seq, max(caps), status=st)
+        ref = oracle.decode_step(to_np(qn), to_np(kn), to_np(vn), ko, vo, o_off, seqo, Hkv)
+        check_attention(to_np(out), ref, torch.bfloat16)
+        assert np.array_equal(seq.cpu().numpy(), seqo)
+    assert st.item() == 0
+    # the appended rows went into the caches bit for bit
+    kh, vh = kc_d.float().cpu().numpy(), vc_d.float().cpu().numpy()
+    for b in range(B):
+        at = (rows_of(b, lens[b] + steps)[:, None] + np.arange(row)[None, :]).reshape(-1)
+        assert np.array_equal(kh[at], ko[o_off[b]: o_off[b] + (lens[b] + steps) * row])
+        assert np.array_equal(vh[at], vo[o_off[b]: o_off[b] + (lens[b] + steps) * row])
