@@ -349,6 +349,61 @@ def long_video_benchmark(z, dev, peaks, reps=10, taus=(0.95, 0.99), sustained=25
     return res
 
 
+def long_context_benchmark(z, dev, peaks, lengths=(32768, 131072), H=40, d=128, tau=0.97):
+    """The LLaVA-Next-13B-shaped layer (40 heads x 128) at the long input lengths of the paper's
+    latency table (32K and 128K tokens; inputs drawn on the device): score, select and the sparse
+    prefill, next to the same attention kernel over ALL tokens (tau = 1: what dense causal
+    attention costs here), so the attention's share of the method's prefill speed-up can be read
+    off.  A launch takes 5 to 180 ms, so every figure is under the power cap: fractions are of
+    the sustained bf16 peak."""
+    from paper_2410_08584_b200 import workloads as W
+    res = []
+    for L in lengths:
+        lay = W.heavy_key_layer(L_visual=L - 64, L_text=64, H=H, d=d, tau=tau, seed=BASE_SEED + 40 + L // 1024,
+                                name="llava_next_13b_long", device="cuda")
+        q, k, v, probe = (t.to(dev) for t in (lay.q, lay.k, lay.v, lay.probe_pos))
+        desc = z.layer_desc(q, k)
+        st = torch.zeros(1, dtype=torch.int32, device=dev)
+        acc, norm = z.zipvl_score(desc, q, k, probe, status=st)
+        k_dev, idx = z.zipvl_select(acc, norm, tau, status=st)
+        k_all, idx_all = z.zipvl_select(acc, norm, 1.0, status=st)
+        kk = int(k_dev.item())
+        out = torch.empty_like(q)
+        ws_pf = z.workspace(z.zipvl_workspace_bytes(z.OP_SPARSE_PREFILL, desc), dev)
+
+        def timeit(f, reps):
+            f()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(reps):
+                f()
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) / reps
+
+        reps = 8 if L <= 65536 else 3
+        t_score = timeit(lambda: z.zipvl_score(desc, q, k, probe, acc=acc, norm=norm, status=st), 5)
+        t_sel = timeit(lambda: z.zipvl_select(acc, norm, tau, k_out=k_dev, idx=idx, status=st), 5)
+        t_dense = timeit(lambda: z.zipvl_sparse_prefill(desc, q, k, v, idx_all, k_all, L, out=out, ws=ws_pf,
+                                                        status=st), reps)
+        t_pf = timeit(lambda: z.zipvl_sparse_prefill(desc, q, k, v, idx, k_dev, L, out=out, ws=ws_pf,
+                                                     status=st), reps)
+        chk = check_prefill_rows(lay.q, lay.k, lay.v, idx, k_dev, out, n_rows=12, seed=L)
+        flops = 4.0 * d * H * kk * (kk + 1) / 2.0
+        flops_all = 4.0 * d * H * L * (L + 1) / 2.0
+        res.append({"L": L, "heads": H, "tau": tau, "k": kk, "k_over_L": kk / L, "score_ms": t_score,
+                    "select_ms": t_sel, "sparse_prefill_ms": t_pf,
+                    "prefill_tflops": flops / (t_pf * 1e-3) / 1e12,
+                    "frac_of_bf16_peak": flops / (t_pf * 1e-3) / 1e12 / peaks["tf_sust"],
+                    "all_tokens_ms": t_dense, "all_tokens_tflops": flops_all / (t_dense * 1e-3) / 1e12,
+                    "attention_speedup_vs_all_tokens": t_dense / (t_score + t_sel + t_pf),
+                    "check": chk, "device_status_word": int(st.item())})
+        del q, k, v, out, lay
+        torch.cuda.empty_cache()
+    return res
+
+
 def library_context(z, dev, reps=20):
     """Context rows, not the product: Algorithm 1 the way the paper runs it -- library gathers
     of Q[T], K[T], V[T], an off-the-shelf causal attention kernel on the gathered copies,
@@ -955,6 +1010,13 @@ def run_ours(args, rank, world, local):
         except Exception as e:  # report, never hide
             video = {"error": repr(e)}
 
+    long_ctx = None
+    if not args.no_long_context and not args.no_long_video:
+        try:
+            long_ctx = long_context_benchmark(z, dev, peaks)
+        except Exception as e:  # report, never hide
+            long_ctx = {"error": repr(e)}
+
     # ---- CPU baseline: the oracle on a bounded sample ------------------------------
     cpu = None
     if not args.no_cpu_baseline:
@@ -992,7 +1054,7 @@ def run_ours(args, rank, world, local):
         "graph_replay_ms_per_step": graph_ms,
         "prefill_ms": float(call_ms[0] + call_ms[1] + call_ms[2]),
         "prefill_tflops_selected": flops / (float(call_ms[0] + call_ms[1] + call_ms[2]) * 1e-3) / 1e12,
-        "roofline": roof, "other_kernels": others, "decode": dec, "decode_gqa": dec_gqa, "batched": batched, "kv_quant": quant, "stack": stack, "long_video": video, "library_context": context,
+        "roofline": roof, "other_kernels": others, "decode": dec, "decode_gqa": dec_gqa, "batched": batched, "kv_quant": quant, "stack": stack, "long_video": video, "long_context": long_ctx, "library_context": context,
         "cpu_baseline": cpu,
         "e2e": {"value": e2e_ms / world, "unit": "ms", "h2d_bytes_per_step": int(h2d),
                 "d2h_bytes_per_step": int(d2h),
@@ -1021,6 +1083,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-long-video", action="store_true", help="skip the long-video (18K-token GQA) leg")
     ap.add_argument("--no-batched", action="store_true", help="skip the 4-sequences-per-call leg")
+    ap.add_argument("--no-long-context", action="store_true", help="skip the 32K / 128K-token leg")
     ap.add_argument("--min-region-ms", type=float, default=MIN_REGION_MS,
                     help="the K-step loop is repeated until the timed region spans this long (0: K steps only, for profiler runs)")
     ap.add_argument("--only-long-video", action="store_true",

@@ -84,6 +84,15 @@ def test_llava_next_13b_stack_all_forty_layers(zipvl):
     assert len(set(ks)) >= 30 and max(ks) > 3 * min(ks), f"per-layer k should vary widely: {ks}"
 
 
+def test_llava_next_13b_layer_at_32k_tokens(zipvl):
+    """The 13B-shaped layer at the first of the long input lengths the bench's long-context leg
+    times (32768 tokens, 40 heads x 128): scores in full, the selection exactly, sampled rows
+    of the attention, compaction and the fused call."""
+    layer = W.heavy_key_layer(L_visual=32768 - 64, L_text=64, H=40, seed=W.BASE_SEED + 72, name="llava_next_13b_long")
+    k = run_layer(zipvl, layer, n_rows=12, seed=3)
+    assert 0.5 * layer.L < k < layer.L
+
+
 def test_full_size_layer_repeated_on_a_side_stream(zipvl):
     """The whole chain (score, select, fused attention + compaction) three hundred times on a
     non-default stream, where every launch is a programmatic dependent of the one before
