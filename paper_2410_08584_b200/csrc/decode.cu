@@ -281,8 +281,11 @@ __device__ __forceinline__ void store2(__nv_bfloat16 *p, float a, float b) {
 }
 __device__ __forceinline__ void store2(__half *p, float a, float b) { *reinterpret_cast<__half2 *>(p) = __floats2half2_rn(a, b); }
 
-template <typename T, int D>
-__global__ void __launch_bounds__(256)
+// kMergeUnroll: slots per lane in flight.  8 behind the CUDA-core kernel; 6 behind the tensor-core
+// kernels, which keeps the merge at 48 registers: its CTAs then fit beside a persistent decode CTA
+// (544 threads x 96 registers) and wait there, staged, while that kernel runs.
+template <typename T, int D, int kMergeUnroll>
+__global__ void __launch_bounds__(256, kMergeUnroll == 8 ? 4 : 5)
 decode_merge_kernel(int Hq, int lanes, int n_chunks, const float *__restrict__ ws,
                     const int *__restrict__ lens, int32_t *__restrict__ seq_lens, T *__restrict__ out,
                     const int *__restrict__ used, int group) {
@@ -298,10 +301,10 @@ decode_merge_kernel(int Hq, int lanes, int n_chunks, const float *__restrict__ w
     // the tensor-core kernel fills only the first used[request, kv head] slots of a head
     const int n_used = used ? min(n_chunks, max(0, used[b * (Hq / group) + hq / group])) : n_chunks;
     float M = -INFINITY, Ls = 0.f, O0 = 0.f, O1 = 0.f;
-    for (int i0 = part; i0 < n_used; i0 += 8 * lanes) {
-        float2 ml[8], oi[8];
+    for (int i0 = part; i0 < n_used; i0 += kMergeUnroll * lanes) {
+        float2 ml[kMergeUnroll], oi[kMergeUnroll];
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
+        for (int u = 0; u < kMergeUnroll; ++u) {
             const int i = i0 + u * lanes;
             const bool in = live && i < n_used;
             const float *p = src + (long long)(in ? i : 0) * (D + 2);   // (a slot is (D + 2) * 4 bytes: 8-byte aligned)
@@ -309,7 +312,7 @@ decode_merge_kernel(int Hq, int lanes, int n_chunks, const float *__restrict__ w
             oi[u] = in ? __ldcg(reinterpret_cast<const float2 *>(p + 2 + c)) : make_float2(0.f, 0.f);
         }
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
+        for (int u = 0; u < kMergeUnroll; ++u) {
             if (ml[u].x != -INFINITY) {
                 const float Mn = fmaxf(M, ml[u].x);
                 const float wo = fast_exp2(M - Mn), wn = fast_exp2(ml[u].x - Mn);
@@ -416,7 +419,7 @@ zipvl_status run(const zipvl_decode_desc &d, float scale_log2, const void *q, co
 #undef ZIPVL_DEC_P
     if (le == cudaSuccess) {
         const int lanes = merge_lanes(B, Hq, D, n_chunks);
-        le = launch_dependent(decode_merge_kernel<T, D>, merge_grid(B, Hq, D, lanes), dim3(256), 0, st, Hq,
+        le = launch_dependent(decode_merge_kernel<T, D, 8>, merge_grid(B, Hq, D, lanes), dim3(256), 0, st, Hq,
                               lanes, n_chunks, (const float *)wsf, (const int *)lens, seq_lens, (T *)out,
                               (const int *)nullptr, 1);
     }
@@ -439,7 +442,7 @@ zipvl_status launch_decode_merge(int dtype, int D, int Hq, int B, int chunk, int
     const int lanes = merge_lanes(B, Hq, D, n_chunks);
     const dim3 grid = merge_grid(B, Hq, D, lanes);
 #define ZIPVL_MERGE(T_, D_) \
-    le = launch_dependent(decode_merge_kernel<T_, D_>, grid, dim3(256), 0, st, Hq, lanes, n_chunks, ws, lens, seq_lens, (T_ *)out, used, group)
+    le = launch_dependent(decode_merge_kernel<T_, D_, 6>, grid, dim3(256), 0, st, Hq, lanes, n_chunks, ws, lens, seq_lens, (T_ *)out, used, group)
     if (dtype == ZIPVL_BF16 && D == 128) ZIPVL_MERGE(__nv_bfloat16, 128);
     else if (dtype == ZIPVL_BF16 && D == 96) ZIPVL_MERGE(__nv_bfloat16, 96);
     else if (dtype == ZIPVL_BF16 && D == 64) ZIPVL_MERGE(__nv_bfloat16, 64);
