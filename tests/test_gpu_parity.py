@@ -836,6 +836,11 @@ def test_decode_kernel_choice_can_be_forced_and_both_match_the_oracle(zipvl, mon
     ("tcp", 1500, 12, 4),      # far more (request, kv head) pairs than CTAs: dozens of segments per CTA
     ("tc", 700, 8, 2),
     ("simt", 700, 8, 8),
+    # batch sizes at which the merge kernel runs with four and with two lanes per head (eight in
+    # the small batches of the other tests, one in the large ones above)
+    ("tcp", 40, 28, 4),
+    ("tc", 80, 28, 4),
+    ("simt", 40, 32, 32),
 ])
 def test_decode_on_many_short_requests(zipvl, monkeypatch, kernel, B, Hq, Hkv):
     """Hundreds of requests of zero to a few hundred rows, a few long ones among them, one step with
