@@ -316,3 +316,48 @@ def test_grouped_query_decode_full_size(zipvl, paged):
         at = (rows_of(b, lens[b] + steps)[:, None] + np.arange(row)[None, :]).reshape(-1)
         assert np.array_equal(kh[at], ko[o_off[b]: o_off[b] + (lens[b] + steps) * row])
         assert np.array_equal(vh[at], vo[o_off[b]: o_off[b] + (lens[b] + steps) * row])
+
+
+@pytest.mark.parametrize("kernel", ["tc", "tcp"])
+def test_grouped_query_decode_many_steps_on_a_side_stream(zipvl, monkeypatch, kernel):
+    """Two hundred decode steps with appends per shape on a non-default stream, every launch a
+    programmatic dependent of the one before, on both tensor-core kernels: no wait runs out (status
+    word), the lengths advance by one per step, and the last step's output matches the oracle."""
+    z = zipvl
+    monkeypatch.setenv("ZIPVL_DECODE_KERNEL", kernel)
+    rng = np.random.default_rng(11)
+    for trial, (Hq, Hkv, d) in enumerate([(28, 4, 128), (32, 2, 64), (16, 8, 96)]):
+        B, steps = int(rng.integers(3, 12)), 200
+        lens = [int(x) for x in rng.integers(0, 5000, B)]
+        row = Hkv * d
+        caps = [n + steps for n in lens]
+        g = torch.Generator().manual_seed(trial)
+        kc = torch.randn(sum(caps) * row, generator=g).to(torch.bfloat16)
+        vc = torch.randn(sum(caps) * row, generator=g).to(torch.bfloat16)
+        off = np.concatenate([[0], np.cumsum([c * row for c in caps[:-1]])]).astype(np.int64)
+        q = torch.randn(B, Hq, d, generator=g).to(torch.bfloat16)
+        kn = torch.randn(B, Hkv, d, generator=g).to(torch.bfloat16)
+        vn = torch.randn(B, Hkv, d, generator=g).to(torch.bfloat16)
+        kc_d, vc_d, q_d, kn_d, vn_d = (t.to(DEV) for t in (kc, vc, q, kn, vn))
+        off_d = torch.from_numpy(off).to(DEV)
+        capt = torch.tensor(caps, dtype=torch.int32, device=DEV)
+        seq = torch.tensor(lens, dtype=torch.int32, device=DEV)
+        desc = z.zipvl_decode_desc(B, Hq, Hkv, d, z.ZIPVL_BF16, 0.0)
+        lay = z.zipvl_layer(max(caps), Hq, Hkv, d, z.ZIPVL_BF16, 0, 0, 0, 0.0, 0)
+        ws = z.workspace(z.zipvl_workspace_bytes(z.OP_DECODE, lay, 0, B), DEV)
+        out = torch.empty_like(q_d)
+        st = torch.zeros(1, dtype=torch.int32, device=DEV)
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            for _ in range(steps):
+                z.zipvl_decode(desc, q_d, kn_d, vn_d, kc_d, vc_d, off_d, capt, seq, max(caps), out=out, ws=ws,
+                               status=st)
+        side.synchronize()
+        assert st.item() == 0
+        assert np.array_equal(seq.cpu().numpy(), np.array(lens) + steps)
+        # the oracle's view of the last step: the caches as the GPU left them, one row short
+        ko, vo = kc_d.float().cpu().numpy(), vc_d.float().cpu().numpy()
+        seqo = np.array(lens, np.int32) + steps - 1
+        ref = oracle.decode_step(to_np(q), to_np(kn), to_np(vn), ko, vo, off, seqo, Hkv)
+        check_attention(to_np(out), ref, torch.bfloat16)
