@@ -365,6 +365,31 @@ zipvl_status zipvl_decode_quant(const zipvl_decode_desc *desc, const void *q, co
                                 int32_t *status_word, void *stream);
 
 /*
+ * zipvl_decode_quant_batch -- zipvl_decode_quant for desc->batch requests in one call.
+ * (Algorithm 2, Eq. 4-5 per request; the requests are independent.)
+ * caches: DEVICE array of desc->batch entries, one request's blocks each (all pointers DEVICE,
+ * laid out and aligned as zipvl_decode_quant takes them; lens: that request's int32[2]).
+ * q, out: [batch, Hq, d]; k_new, v_new: [batch, Hkv, d] or both NULL; max_len: host bound on
+ * any request's lens[0] + lens[1] after the append; ws: zipvl_workspace_bytes(ZIPVL_OP_DECODE)
+ * for this batch and L = max_len.  The table lives on the device, so its entries are checked
+ * there: a request whose entry has a NULL or misaligned block, or a capacity below 1, is
+ * skipped (nothing appended, an output of zeros) and reported as ZIPVL_DEV_BAD_INDEX; a full
+ * 4-bit block as ZIPVL_DEV_CAPACITY, per request.  Same shapes as zipvl_decode_quant.
+ * The call enqueues two kernels (three with an append), whatever the batch.
+ */
+typedef struct zipvl_quant_cache {
+    void *k_hi, *v_hi, *params_hi;   /* the 4-bit block */
+    void *k_lo, *v_lo, *params_lo;   /* the 2-bit block */
+    int32_t *lens;                   /* rows in hi, lo */
+    int32_t cap_hi, cap_lo;
+} zipvl_quant_cache;
+
+zipvl_status zipvl_decode_quant_batch(const zipvl_decode_desc *desc, const void *q, const void *k_new,
+                                      const void *v_new, const zipvl_quant_cache *caches, int32_t max_len,
+                                      void *out, void *ws, size_t ws_bytes, int32_t *status_word,
+                                      void *stream);
+
+/*
  * zipvl_decode_noalloc -- zipvl_decode for callers that cannot allocate.
  * (The paper has no counterpart: this is a deployment variant of the decode
  * step, same arithmetic, same kernels.)

@@ -26,7 +26,7 @@ EXPORTS = ["zipvl_status_string", "zipvl_last_error", "zipvl_version", "zipvl_la
            "zipvl_score", "zipvl_select", "zipvl_sparse_prefill", "zipvl_compact_kv",
            "zipvl_sparse_prefill_compact", "zipvl_workspace_bytes_batch", "zipvl_score_batch",
            "zipvl_select_batch", "zipvl_sparse_prefill_batch",
-           "zipvl_decode", "zipvl_decode_paged", "zipvl_quantize_kv", "zipvl_decode_quant", "zipvl_decode_noalloc", "zipvl_prefill_layer_host", "zipvl_layer_step_host",
+           "zipvl_decode", "zipvl_decode_paged", "zipvl_quantize_kv", "zipvl_decode_quant", "zipvl_decode_quant_batch", "zipvl_decode_noalloc", "zipvl_prefill_layer_host", "zipvl_layer_step_host",
            "zipvl_release_host_scratch", "zipvl_selftest_wait_timeout"]
 
 
@@ -108,6 +108,8 @@ def load():
     lib.zipvl_decode_quant.restype = C.c_int
     lib.zipvl_decode_quant.argtypes = [C.POINTER(zipvl_decode_desc), vp, vp, vp, vp, vp, vp, i32, vp, vp, vp, i32,
                                        vp, i32, vp, vp, sz, vp, vp]
+    lib.zipvl_decode_quant_batch.restype = C.c_int
+    lib.zipvl_decode_quant_batch.argtypes = [C.POINTER(zipvl_decode_desc), vp, vp, vp, vp, i32, vp, vp, sz, vp, vp]
     lib.zipvl_decode_noalloc.restype = C.c_int
     lib.zipvl_decode_noalloc.argtypes = [C.POINTER(zipvl_decode_desc), vp, vp, vp, vp, vp, vp, vp,
                                          vp, i32, vp, vp, vp]
@@ -425,6 +427,34 @@ def zipvl_decode_quant(desc, q, k_new, v_new, cache, max_len, out=None, ws=None,
                                      _ptr(cache.v_lo), _ptr(cache.p_lo), cache.cap_lo, _ptr(cache.lens),
                                      int(max_len), _ptr(out), _ptr(ws), ws.numel(), _ptr(status),
                                      _stream(stream)))
+    return out
+
+
+def quant_cache_table(caches, device):
+    """The device table zipvl_decode_quant_batch takes: one 64-byte zipvl_quant_cache entry per
+    request (seven device pointers, then the two capacities)."""
+    rows = []
+    for c in caches:
+        rows.append([c.k_hi.data_ptr(), c.v_hi.data_ptr(), c.p_hi.data_ptr(), c.k_lo.data_ptr(),
+                     c.v_lo.data_ptr(), c.p_lo.data_ptr(), c.lens.data_ptr(),
+                     (int(c.cap_hi) & 0xffffffff) | (int(c.cap_lo) << 32)])
+    return torch.tensor(rows, dtype=torch.int64).to(device)
+
+
+def zipvl_decode_quant_batch(desc, q, k_new, v_new, table, max_len, out=None, ws=None, status=None, stream=None):
+    """One decode step of desc.batch requests over their mixed-precision caches (table:
+    quant_cache_table of the requests' QuantCache objects); returns out [B,Hq,d]."""
+    _dev(q, "q"), _dev(table, "table", torch.int64)
+    if table.shape[0] != desc.batch or table.shape[1] != 8:
+        raise ValueError("table must be int64 [batch, 8]")
+    out = torch.empty_like(q) if out is None else out
+    if ws is None:
+        lay = zipvl_layer(int(max_len), desc.n_q_heads, desc.n_kv_heads, desc.head_dim, desc.dtype,
+                          0, 0, 0, 0.0, 0)
+        ws = workspace(zipvl_workspace_bytes(OP_DECODE, lay, 0, desc.batch), q.device)
+    _check(load().zipvl_decode_quant_batch(C.byref(desc), _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(table),
+                                           int(max_len), _ptr(out), _ptr(ws), ws.numel(), _ptr(status),
+                                           _stream(stream)))
     return out
 
 

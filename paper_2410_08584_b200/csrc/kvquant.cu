@@ -84,6 +84,23 @@ struct QuantBlocks {
     int cap_hi, cap_lo;
 };
 
+// The blocks of request b: the call's own (one request) or entry b of the caller's device table.
+// A table entry cannot be checked on the host: one with a NULL or misaligned block or a capacity
+// below 1 is reported and its request skipped (no append, an output of zeros).
+__device__ __forceinline__ bool request_blocks(const zipvl_quant_cache *caches, int b, QuantBlocks &qb,
+                                               int32_t *&lens) {
+    if (caches == nullptr) return true;
+    const zipvl_quant_cache c = caches[b];
+    qb = QuantBlocks{(unsigned char *)c.k_hi, (unsigned char *)c.v_hi, (unsigned char *)c.k_lo, (unsigned char *)c.v_lo,
+                     (unsigned short *)c.params_hi, (unsigned short *)c.params_lo, c.cap_hi, c.cap_lo};
+    lens = c.lens;
+    const unsigned long long all = (unsigned long long)c.k_hi | (unsigned long long)c.v_hi | (unsigned long long)c.k_lo |
+                                   (unsigned long long)c.v_lo | (unsigned long long)c.params_hi |
+                                   (unsigned long long)c.params_lo;
+    return c.k_hi && c.v_hi && c.k_lo && c.v_lo && c.params_hi && c.params_lo && c.lens && !(all & 15ull) &&
+           !((unsigned long long)c.lens & 3ull) && c.cap_hi >= 1 && c.cap_lo >= 1;
+}
+
 template <bool kHalf, int D>
 __global__ void __launch_bounds__(kQuantThreads)
 quantize_kv_kernel(LayerArgs a, const unsigned short *__restrict__ k, const unsigned short *__restrict__ v,
@@ -163,14 +180,22 @@ quantize_kv_kernel(LayerArgs a, const unsigned short *__restrict__ k, const unsi
 }
 
 // Eq. 4 on the quantised cache: the new token's key and value, quantised at 4 bits, become
-// row lens[0] of the "hi" block; lens[0] += 1.  One CTA, one lane group per KV head.
+// row lens[0] of the "hi" block; lens[0] += 1.  One CTA per request, one lane group per KV head.
 template <bool kHalf, int D>
 __global__ void __launch_bounds__(1024)
 quant_append_kernel(int Hkv, const unsigned short *__restrict__ k_new, const unsigned short *__restrict__ v_new,
-                    QuantBlocks qb, int32_t *__restrict__ lens, int32_t *status_word) {
+                    QuantBlocks qb, int32_t *lens, const zipvl_quant_cache *__restrict__ caches,
+                    int32_t *status_word) {
     constexpr int kLanes = D / 8;
     grid_launch_dependents();
-    grid_dependency_wait(k_new, v_new, lens);
+    grid_dependency_wait(k_new, v_new, lens, caches);
+    const int b = blockIdx.x;
+    if (!request_blocks(caches, b, qb, lens)) {
+        if (threadIdx.x == 0) report(status_word, ZIPVL_DEV_BAD_INDEX);
+        return;
+    }
+    k_new += (long long)b * Hkv * D;
+    v_new += (long long)b * Hkv * D;
     const int n_hi = lens[0];
     const bool room = n_hi >= 0 && n_hi < qb.cap_hi;
     const int grp = threadIdx.x / kLanes, lg = threadIdx.x % kLanes;
@@ -215,15 +240,20 @@ __device__ __forceinline__ float code_to_float(uint32_t c) { return __uint_as_fl
 template <bool kHalf, int D, int GT>
 __global__ void __launch_bounds__(kDqThreads)
 decode_quant_kernel(int Hq, int Hkv, float scale_log2, const unsigned short *__restrict__ q, QuantBlocks qb,
-                    const int32_t *__restrict__ lens, int max_len, int chunk, int n_chunks,
-                    float *__restrict__ ws, int *__restrict__ lens_ws, int32_t *status_word) {
+                    int32_t *lens, const zipvl_quant_cache *__restrict__ caches, int max_len, int chunk,
+                    int n_chunks, float *__restrict__ ws, int *__restrict__ lens_ws, int32_t *status_word) {
     constexpr int CPL = D / kDqLanes;            // channels per lane: 16 or 8
     constexpr int RPW = 32 / kDqLanes;           // rows per warp per load: 4
     constexpr int NG = (kDqThreads / 32) * RPW;  // row groups per CTA: 16
     __shared__ float sm_o[NG][GT][D];
     __shared__ float sm_m[NG][GT], sm_l[NG][GT];
     grid_launch_dependents();
-    grid_dependency_wait(q, lens, qb.k_hi, qb.v_hi, qb.k_lo, qb.v_lo, qb.p_hi, qb.p_lo);
+    grid_dependency_wait(q, lens, caches, qb.k_hi, qb.v_hi, qb.k_lo, qb.v_lo, qb.p_hi, qb.p_lo);
+    const int b = blockIdx.z;                    // request
+    const bool blocks_ok = request_blocks(caches, b, qb, lens);
+    q += (long long)b * Hq * D;
+    ws += (long long)b * Hq * n_chunks * (D + 2);
+    lens_ws += 2 * b;
     const int G = Hq / Hkv;
     const int hkv = blockIdx.y, h0 = hkv * G;
     const int n_heads = min(GT, G);
@@ -249,8 +279,8 @@ decode_quant_kernel(int Hq, int Hkv, float scale_log2, const unsigned short *__r
         for (int o = kDqLanes / 2; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
         qsum[g] = part;
     }
-    int n_hi = lens[0], n_lo = lens[1];
-    const bool bad = n_hi < 0 || n_lo < 0 || n_hi > qb.cap_hi || n_lo > qb.cap_lo;
+    int n_hi = blocks_ok ? lens[0] : 0, n_lo = blocks_ok ? lens[1] : 0;
+    const bool bad = !blocks_ok || n_hi < 0 || n_lo < 0 || n_hi > qb.cap_hi || n_lo > qb.cap_lo;
     if (bad) {
         if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) report(status_word, ZIPVL_DEV_BAD_INDEX);
         n_hi = 0; n_lo = 0;
@@ -412,24 +442,26 @@ zipvl_status run_quantize(const LayerArgs &a, const void *k, const void *v, cons
 
 template <bool kHalf, int D>
 zipvl_status run_decode_quant(const zipvl_decode_desc &d, float scale_log2, const void *q, const void *k_new,
-                              const void *v_new, const QuantBlocks &qb, int32_t *lens, int max_len, void *out,
-                              void *ws, int32_t *status_word, cudaStream_t st) {
-    const int Hq = d.n_q_heads, Hkv = d.n_kv_heads, G = Hq / Hkv;
+                              const void *v_new, const QuantBlocks &qb, int32_t *lens,
+                              const zipvl_quant_cache *caches, int max_len, void *out, void *ws,
+                              int32_t *status_word, cudaStream_t st) {
+    const int Hq = d.n_q_heads, Hkv = d.n_kv_heads, G = Hq / Hkv, B = d.batch;
     cudaError_t e = cudaSuccess;
     if (k_new) {
-        e = launch_dependent(quant_append_kernel<kHalf, D>, dim3(1), dim3(Hkv * (D / 8)), 0, st, Hkv,
-                             (const unsigned short *)k_new, (const unsigned short *)v_new, qb, lens, status_word);
+        e = launch_dependent(quant_append_kernel<kHalf, D>, dim3(B), dim3(Hkv * (D / 8)), 0, st, Hkv,
+                             (const unsigned short *)k_new, (const unsigned short *)v_new, qb, lens, caches,
+                             status_word);
         if (e != cudaSuccess) return fail(ZIPVL_ERR_CUDA, "zipvl_decode_quant: launch: %s", cudaGetErrorString(e));
         count_launches(1);
     }
-    const int chunk = decode_chunk_rows(1, Hq, max_len);
+    const int chunk = decode_chunk_rows(B, Hq, max_len);
     const int n_chunks = (max_len + chunk - 1) / chunk;
     float *wsf = reinterpret_cast<float *>(ws);
-    int *lens_ws = reinterpret_cast<int *>(reinterpret_cast<char *>(ws) + decode_partial_bytes(1, Hq, D, max_len));
-    const dim3 grid(n_chunks, Hkv);
+    int *lens_ws = reinterpret_cast<int *>(reinterpret_cast<char *>(ws) + decode_partial_bytes(B, Hq, D, max_len));
+    const dim3 grid(n_chunks, Hkv, B);
 #define ZIPVL_DQ(GT_)                                                                                       \
     e = launch_dependent(decode_quant_kernel<kHalf, D, GT_>, grid, dim3(kDqThreads), 0, st, Hq, Hkv, scale_log2, \
-                         (const unsigned short *)q, qb, (const int32_t *)lens, max_len, chunk, n_chunks, wsf,    \
+                         (const unsigned short *)q, qb, lens, caches, max_len, chunk, n_chunks, wsf,             \
                          lens_ws, status_word)
     if (G == 1) ZIPVL_DQ(1);
     else if (G == 2) ZIPVL_DQ(2);
@@ -437,7 +469,9 @@ zipvl_status run_decode_quant(const zipvl_decode_desc &d, float scale_log2, cons
 #undef ZIPVL_DQ
     if (e != cudaSuccess) return fail(ZIPVL_ERR_CUDA, "zipvl_decode_quant: launch: %s", cudaGetErrorString(e));
     count_launches(1);
-    return launch_decode_merge(d.dtype, D, Hq, 1, chunk, n_chunks, wsf, lens_ws, lens, out, st);
+    // (the append kernel has counted the new rows: the merge writes no length; the words behind the
+    // (length, appended) pairs stand in for its length array)
+    return launch_decode_merge(d.dtype, D, Hq, B, chunk, n_chunks, wsf, lens_ws, lens_ws + 2 * B, out, st);
 }
 
 }  // namespace
@@ -488,14 +522,10 @@ extern "C" zipvl_status zipvl_quantize_kv(const zipvl_layer *l, const void *k, c
                       : run_quantize<false, 64>(a, k, v, idx, k_dev, k_max, qb, lens_out, status_word, st);
 }
 
-extern "C" zipvl_status zipvl_decode_quant(const zipvl_decode_desc *d, const void *q, const void *k_new,
-                                           const void *v_new, void *k_hi, void *v_hi, void *params_hi,
-                                           int32_t cap_hi, void *k_lo, void *v_lo, void *params_lo,
-                                           int32_t cap_lo, int32_t *lens, int32_t max_len, void *out, void *ws,
-                                           size_t ws_bytes, int32_t *status_word, void *stream) {
-    const char *who = "zipvl_decode_quant";
+// what the two decode entries check alike
+static zipvl_status check_decode_quant(const char *who, const zipvl_decode_desc *d, const void *q, const void *k_new,
+                                       const void *v_new, int max_len, const void *out, const void *ws) {
     if (!d) return fail(ZIPVL_ERR_INVALID_ARG, "%s: desc is NULL", who);
-    if (d->batch != 1) return fail(ZIPVL_ERR_UNSUPPORTED, "%s: batch %d (one request per call)", who, d->batch);
     if (d->n_q_heads < 1 || d->n_kv_heads < 1 || d->n_q_heads % d->n_kv_heads)
         return fail(ZIPVL_ERR_INVALID_ARG, "%s: heads %d / %d", who, d->n_q_heads, d->n_kv_heads);
     const int G = d->n_q_heads / d->n_kv_heads;
@@ -503,23 +533,60 @@ extern "C" zipvl_status zipvl_decode_quant(const zipvl_decode_desc *d, const voi
         (G != 1 && G != 2 && G != 4))
         return fail(ZIPVL_ERR_UNSUPPORTED, "%s: dtype %d head_dim %d group %d (16-bit storage, head_dim 64 or 128, "
                     "1, 2 or 4 query heads per KV head)", who, d->dtype, d->head_dim, G);
-    if (!q || !lens || !out || !ws) return fail(ZIPVL_ERR_INVALID_ARG, "%s: NULL pointer", who);
+    if (!q || !out || !ws) return fail(ZIPVL_ERR_INVALID_ARG, "%s: NULL pointer", who);
     if ((k_new == NULL) != (v_new == NULL))
         return fail(ZIPVL_ERR_INVALID_ARG, "%s: k_new and v_new must both be given or both NULL", who);
     if (max_len < 1) return fail(ZIPVL_ERR_INVALID_ARG, "%s: max_len = %d", who, max_len);
     if (!(d->softmax_scale >= 0.f) || isinf(d->softmax_scale)) return fail(ZIPVL_ERR_INVALID_ARG, "%s: softmax_scale", who);
     if (((uintptr_t)q | (uintptr_t)out | (uintptr_t)ws | (uintptr_t)k_new | (uintptr_t)v_new) & 15u)
         return fail(ZIPVL_ERR_INVALID_ARG, "%s: tensors must be 16-byte aligned", who);
+    return ZIPVL_OK;
+}
+
+static zipvl_status dispatch_decode_quant(const zipvl_decode_desc &d, float scale, const void *q, const void *k_new,
+                                          const void *v_new, const QuantBlocks &qb, int32_t *lens,
+                                          const zipvl_quant_cache *caches, int max_len, void *out, void *ws,
+                                          int32_t *status_word, cudaStream_t st) {
+    const bool half = d.dtype == ZIPVL_F16;
+    if (half) return d.head_dim == 128 ? run_decode_quant<true, 128>(d, scale, q, k_new, v_new, qb, lens, caches, max_len, out, ws, status_word, st)
+                                       : run_decode_quant<true, 64>(d, scale, q, k_new, v_new, qb, lens, caches, max_len, out, ws, status_word, st);
+    return d.head_dim == 128 ? run_decode_quant<false, 128>(d, scale, q, k_new, v_new, qb, lens, caches, max_len, out, ws, status_word, st)
+                             : run_decode_quant<false, 64>(d, scale, q, k_new, v_new, qb, lens, caches, max_len, out, ws, status_word, st);
+}
+
+extern "C" zipvl_status zipvl_decode_quant(const zipvl_decode_desc *d, const void *q, const void *k_new,
+                                           const void *v_new, void *k_hi, void *v_hi, void *params_hi,
+                                           int32_t cap_hi, void *k_lo, void *v_lo, void *params_lo,
+                                           int32_t cap_lo, int32_t *lens, int32_t max_len, void *out, void *ws,
+                                           size_t ws_bytes, int32_t *status_word, void *stream) {
+    const char *who = "zipvl_decode_quant";
+    const zipvl_status sv = check_decode_quant(who, d, q, k_new, v_new, max_len, out, ws);
+    if (sv != ZIPVL_OK) return sv;
+    if (d->batch != 1) return fail(ZIPVL_ERR_UNSUPPORTED, "%s: batch %d (one request per call)", who, d->batch);
+    if (!lens) return fail(ZIPVL_ERR_INVALID_ARG, "%s: NULL pointer", who);
     QuantBlocks qb;
     const zipvl_status s = check_blocks(who, d->n_kv_heads, k_hi, v_hi, params_hi, cap_hi, k_lo, v_lo, params_lo, cap_lo, &qb);
     if (s != ZIPVL_OK) return s;
     const size_t need = (decode_ws_bytes(1, d->n_q_heads, d->head_dim, max_len) + 255) & ~(size_t)255;
     if (ws_bytes < need) return fail(ZIPVL_ERR_WORKSPACE, "%s: workspace %zu < %zu", who, ws_bytes, need);
     const float scale = (d->softmax_scale > 0.f ? d->softmax_scale : 1.0f / sqrtf((float)d->head_dim)) * kLog2e;
-    cudaStream_t st = (cudaStream_t)stream;
-    const bool half = d->dtype == ZIPVL_F16;
-    if (half) return d->head_dim == 128 ? run_decode_quant<true, 128>(*d, scale, q, k_new, v_new, qb, lens, max_len, out, ws, status_word, st)
-                                        : run_decode_quant<true, 64>(*d, scale, q, k_new, v_new, qb, lens, max_len, out, ws, status_word, st);
-    return d->head_dim == 128 ? run_decode_quant<false, 128>(*d, scale, q, k_new, v_new, qb, lens, max_len, out, ws, status_word, st)
-                              : run_decode_quant<false, 64>(*d, scale, q, k_new, v_new, qb, lens, max_len, out, ws, status_word, st);
+    return dispatch_decode_quant(*d, scale, q, k_new, v_new, qb, lens, nullptr, max_len, out, ws, status_word,
+                                 (cudaStream_t)stream);
+}
+
+extern "C" zipvl_status zipvl_decode_quant_batch(const zipvl_decode_desc *d, const void *q, const void *k_new,
+                                                 const void *v_new, const zipvl_quant_cache *caches,
+                                                 int32_t max_len, void *out, void *ws, size_t ws_bytes,
+                                                 int32_t *status_word, void *stream) {
+    const char *who = "zipvl_decode_quant_batch";
+    const zipvl_status s = check_decode_quant(who, d, q, k_new, v_new, max_len, out, ws);
+    if (s != ZIPVL_OK) return s;
+    if (d->batch < 1 || d->batch > 65535) return fail(ZIPVL_ERR_INVALID_ARG, "%s: batch %d not in [1, 65535]", who, d->batch);
+    if (d->n_kv_heads > 1024 / 16) return fail(ZIPVL_ERR_UNSUPPORTED, "%s: more than 64 KV heads", who);
+    if (!caches || ((uintptr_t)caches & 7u)) return fail(ZIPVL_ERR_INVALID_ARG, "%s: caches is NULL or misaligned", who);
+    const size_t need = (decode_ws_bytes(d->batch, d->n_q_heads, d->head_dim, max_len) + 255) & ~(size_t)255;
+    if (ws_bytes < need) return fail(ZIPVL_ERR_WORKSPACE, "%s: workspace %zu < %zu", who, ws_bytes, need);
+    const float scale = (d->softmax_scale > 0.f ? d->softmax_scale : 1.0f / sqrtf((float)d->head_dim)) * kLog2e;
+    return dispatch_decode_quant(*d, scale, q, k_new, v_new, QuantBlocks{}, nullptr, caches, max_len, out, ws, status_word,
+                                 (cudaStream_t)stream);
 }

@@ -135,6 +135,13 @@ def test_argument_validation_without_a_device(lib):
     assert dq(C.byref(d1), p, None, None, p, p, p, 8, p, p, p, 8, p, 16, p, p, 8, None, None) == 3
     d3 = z.zipvl_decode_desc(1, 6, 2, 64, 0, 0.0)
     assert dq(C.byref(d3), p, None, None, p, p, p, 8, p, p, p, 8, p, 16, p, p, 1 << 20, None, None) == 2  # 3 heads per KV head
+    # ... and its batched form: the table, the workspace for the whole batch, the same shapes
+    dqb = lib.zipvl_decode_quant_batch
+    assert dqb(C.byref(d), p, None, None, null, 16, p, p, 1 << 20, None, None) == 1             # no table
+    assert dqb(C.byref(d), p, None, None, C.c_void_p(0x1004), 16, p, p, 1 << 20, None, None) == 1
+    assert dqb(C.byref(d), p, p, None, p, 16, p, p, 1 << 20, None, None) == 1                   # k_new without v_new
+    assert dqb(C.byref(d), p, None, None, p, 16, p, p, 8, None, None) == 3
+    assert dqb(C.byref(d3), p, None, None, p, 16, p, p, 1 << 20, None, None) == 2               # 3 heads per KV head
     # the wait self-test: limits outside [1, 2^20] and a missing status word are refused
     assert lib.zipvl_selftest_wait_timeout(0, None, p, None) == 1
     assert lib.zipvl_selftest_wait_timeout(1 << 21, None, p, None) == 1
