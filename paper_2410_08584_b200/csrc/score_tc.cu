@@ -290,9 +290,13 @@ score_tc_kernel(const __grid_constant__ CUtensorMap kmap, LayerArgs a,
                     }
                     first_vis = lo;
                 }
+                // probes below the warp's first key see none of its keys: whole 32-probe chunks of
+                // them are left out (probes ascend, the warp's rows too: lane 0 has the smallest bound)
+                const int first_vis_warp = __shfl_sync(0xffffffffu, first_vis, 0);
                 float cs4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                for (int c = 0; c < 4; ++c)
+                for (int c = 0; c < 4; ++c) {
+                    if ((c + 1) * 32 <= first_vis_warp) continue;
 #pragma unroll
                     for (int e = 0; e < 32; ++e) {
                         const int pr = c * 32 + e;
@@ -300,6 +304,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap kmap, LayerArgs a,
                         const float p = ex2(fmaf(__uint_as_float(sr[c][e]), a.scale_log2, sNegM[pr])) * sIl[pr];
                         cs4[e & 3] += (pr >= first_vis) ? p : 0.f;
                     }
+                }
                 if (j < a.L) partial[(long long)h * a.L + j] = (cs4[0] + cs4[1]) + (cs4[2] + cs4[3]);
             }
         }
