@@ -15,8 +15,9 @@
 // map over K as [L, Hkv*d], 128-byte swizzle, two 64-column boxes per tile) into
 // a two-deep ring; one thread issues tcgen05.mma into one of two TMEM buffers so
 // the next tile's MMA overlaps the current tile's exponentials.
-// The last CTA to finish a key chunk sums the heads in fixed order and
-// normalises -- no float atomics anywhere, so results repeat bit for bit.
+// Every head adds its column sums to 64-bit fixed-point totals (integer adds: no order to
+// depend on, so results repeat bit for bit); the last CTA to finish a key chunk turns the
+// totals into floats and normalises.
 #include <cuda.h>
 
 #include "tc.cuh"
@@ -34,6 +35,7 @@ constexpr int kHalfBytes = 128 * 128;
 constexpr int kTileBytes = 2 * kHalfBytes;
 constexpr int kKStages = 2;
 constexpr int kThreadsSc = 192;
+constexpr float kFxScale = 1099511627776.0f;   // 2^40: units of the fixed-point column totals
 constexpr uint32_t kTmemColsSc = 256;
 
 struct ScBarriers {
@@ -70,7 +72,7 @@ __global__ void __launch_bounds__(kThreadsSc, 2)   // two CTAs per SM hide each 
 score_tc_kernel(const __grid_constant__ CUtensorMap kmap, LayerArgs a,
                 const __nv_bfloat16 *__restrict__ q, const int32_t *__restrict__ probe_pos, int P,
                 int tiles_per_chunk, int n_chunks, float2 *__restrict__ stats,
-                float *__restrict__ partial, int *__restrict__ counters,
+                unsigned long long *__restrict__ accfx, int *__restrict__ counters,
                 float *__restrict__ acc, float *__restrict__ norm, int32_t *status_word) {
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -83,13 +85,13 @@ score_tc_kernel(const __grid_constant__ CUtensorMap kmap, LayerArgs a,
     ScBarriers *bar = reinterpret_cast<ScBarriers *>(sPos + kMaxProbe);
     volatile int *abort_flag = &bar->abort_flag;
 
-    // blockIdx.z = sequence of a batch: its own probe rows, statistics, partial sums, counters
+    // blockIdx.z = sequence of a batch: its own probe rows, statistics, column totals, counters
     // and scores, stacked; K of all sequences is one tensor map of n_seq * L rows
     const int chunk = blockIdx.x, h = blockIdx.y, g = h / a.G, z = blockIdx.z;
     q += z * a.q_seq;
     probe_pos += (long long)z * P;
     stats += (long long)z * a.Hq * n_chunks * kMaxProbe;
-    partial += (long long)z * a.Hq * a.L;
+    accfx += (long long)z * a.L;
     counters += z * n_chunks;
     acc += (long long)z * a.L;
     norm += (long long)z * a.L;
@@ -305,7 +307,11 @@ score_tc_kernel(const __grid_constant__ CUtensorMap kmap, LayerArgs a,
                         cs4[e & 3] += (pr >= first_vis) ? p : 0.f;
                     }
                 }
-                if (j < a.L) partial[(long long)h * a.L + j] = (cs4[0] + cs4[1]) + (cs4[2] + cs4[3]);
+                // the head's column sum goes into the column's fixed-point total (2^-40 units: a sum
+                // of 128 probabilities per head stays far below 2^63): integer adds commute, so the
+                // total does not depend on the order in which the heads arrive
+                if (j < a.L)
+                    atomicAdd(accfx + j, __float2ull_rn(((cs4[0] + cs4[1]) + (cs4[2] + cs4[3])) * kFxScale));
             }
         }
         if (MODE == 0)
@@ -323,11 +329,15 @@ score_tc_kernel(const __grid_constant__ CUtensorMap kmap, LayerArgs a,
         tmem_dealloc(tmem, kTmemColsSc);
     }
     if (MODE == 0) {
-        // arm the per-chunk counter the column-sum kernel uses to find its last CTA
-        if (h == 0 && threadIdx.x == 0) counters[chunk] = 0;
+        // arm the per-chunk counter the column-sum kernel uses to find its last CTA, and clear
+        // the chunk's column totals
+        if (h == 0) {
+            if (threadIdx.x == 0) counters[chunk] = 0;
+            for (int j = t0 * kTile + (int)threadIdx.x; j < min(a.L, t1 * kTile); j += kThreadsSc) accfx[j] = 0ull;
+        }
     } else {
-        // The last head to finish a key chunk sums the heads in fixed order (Eq. 6),
-        // normalises (Eq. 8) and writes the scores: no extra launch, no float atomics.
+        // The last head to finish a key chunk reads the totals of all heads (Eq. 6), normalises
+        // (Eq. 8) and writes the scores: no extra launch, no float atomics.
         __shared__ int is_last;
         if (threadIdx.x == 0) {
             __threadfence();
@@ -349,19 +359,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap kmap, LayerArgs a,
                 n_valid_probes = lo;
             }
             for (int j = jlo + (int)threadIdx.x; j < jhi; j += kThreadsSc) {
-                // heads are added in ascending order (fixed, so the result repeats bit for
-                // bit); up to 32 loads are in flight at a time
-                float sum = 0.f;
-                const float *pj = partial + j;
-                for (int h0 = 0; h0 < a.Hq; h0 += 32) {
-                    float t[32];
-#pragma unroll
-                    for (int u = 0; u < 32; ++u)
-                        t[u] = (h0 + u < a.Hq) ? __ldcg(pj + (long long)(h0 + u) * a.L) : 0.f;
-#pragma unroll
-                    for (int u = 0; u < 32; ++u)
-                        if (h0 + u < a.Hq) sum += t[u];
-                }
+                // the exact total of the heads' sums, rounded once
+                const float sum = (float)((double)__ldcg(accfx + j) * (1.0 / (double)kFxScale));
                 int lo = 0, hi = n_valid_probes;
                 while (lo < hi) {
                     const int mid = (lo + hi) >> 1;
@@ -419,8 +418,8 @@ size_t score_tc_ws_bytes(int L, int Hq, int, int, int n_seq) {
     size_t stats = (size_t)Hq * n_chunks * kMaxProbe * sizeof(float2);
     stats = (stats + 255) & ~(size_t)255;
     stats = ((stats * n_seq) + 255) & ~(size_t)255;
-    const size_t partial = ((size_t)n_seq * Hq * L * sizeof(float) + 255) & ~(size_t)255;
-    return stats + partial + n_seq * n_chunks * sizeof(int);
+    const size_t totals = ((size_t)n_seq * L * sizeof(unsigned long long) + 255) & ~(size_t)255;
+    return stats + totals + n_seq * n_chunks * sizeof(int);
 }
 
 zipvl_status launch_score_tc(const LayerArgs &a, const void *q, const void *k,
@@ -432,9 +431,9 @@ zipvl_status launch_score_tc(const LayerArgs &a, const void *q, const void *k,
     size_t stats_bytes = (size_t)a.n_seq * a.Hq * n_chunks * kMaxProbe * sizeof(float2);
     stats_bytes = (stats_bytes + 255) & ~(size_t)255;
     float2 *stats = reinterpret_cast<float2 *>(ws);
-    float *partial = reinterpret_cast<float *>(reinterpret_cast<char *>(ws) + stats_bytes);
-    const size_t partial_bytes = ((size_t)a.n_seq * a.Hq * a.L * sizeof(float) + 255) & ~(size_t)255;
-    int *counters = reinterpret_cast<int *>(reinterpret_cast<char *>(ws) + stats_bytes + partial_bytes);
+    unsigned long long *accfx = reinterpret_cast<unsigned long long *>(reinterpret_cast<char *>(ws) + stats_bytes);
+    const size_t totals_bytes = ((size_t)a.n_seq * a.L * sizeof(unsigned long long) + 255) & ~(size_t)255;
+    int *counters = reinterpret_cast<int *>(reinterpret_cast<char *>(ws) + stats_bytes + totals_bytes);
 
     // tensor map over K viewed as [L rows, Hkv*d columns], box = 64 columns x 128 rows
     CUtensorMap kmap;
@@ -462,10 +461,10 @@ zipvl_status launch_score_tc(const LayerArgs &a, const void *q, const void *k,
             e = cudaFuncSetAttribute(score_tc_kernel<1, HD_>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kScSmem); \
         if (e != cudaSuccess) return fail(ZIPVL_ERR_CUDA, "score: smem opt-in: %s", cudaGetErrorString(e)); \
         e = launch_dependent(score_tc_kernel<0, HD_>, grid, dim3(kThreadsSc), kScSmem, st, kmap, a, qb, probe_pos, P, \
-                             tpc, n_chunks, stats, partial, counters, acc, norm, status_word);       \
+                             tpc, n_chunks, stats, accfx, counters, acc, norm, status_word);       \
         if (e == cudaSuccess)                                                                        \
             e = launch_dependent(score_tc_kernel<1, HD_>, grid, dim3(kThreadsSc), kScSmem, st, kmap, a, qb, probe_pos, \
-                                 P, tpc, n_chunks, stats, partial, counters, acc, norm, status_word); \
+                                 P, tpc, n_chunks, stats, accfx, counters, acc, norm, status_word); \
     }
     if (a.D == 128) ZIPVL_SCORE_LAUNCH(128)
     else if (a.D == 96) ZIPVL_SCORE_LAUNCH(96)
