@@ -310,8 +310,13 @@ score_tc_kernel(const __grid_constant__ CUtensorMap kmap, LayerArgs a,
                 // the head's column sum goes into the column's fixed-point total (2^-40 units: a sum
                 // of 128 probabilities per head stays far below 2^63): integer adds commute, so the
                 // total does not depend on the order in which the heads arrive
-                if (j < a.L)
-                    atomicAdd(accfx + j, __float2ull_rn(((cs4[0] + cs4[1]) + (cs4[2] + cs4[3])) * kFxScale));
+                // (a sum that is not a number -- a NaN in a query or key row -- sets the total's top
+                // bit, which no sum of the heads reaches: the column's scores come out as NaN)
+                if (j < a.L) {
+                    const float cs = (cs4[0] + cs4[1]) + (cs4[2] + cs4[3]);
+                    if (cs == cs) atomicAdd(accfx + j, __float2ull_rn(cs * kFxScale));
+                    else atomicOr(accfx + j, 1ull << 63);
+                }
             }
         }
         if (MODE == 0)
@@ -360,7 +365,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap kmap, LayerArgs a,
             }
             for (int j = jlo + (int)threadIdx.x; j < jhi; j += kThreadsSc) {
                 // the exact total of the heads' sums, rounded once
-                const float sum = (float)((double)__ldcg(accfx + j) * (1.0 / (double)kFxScale));
+                const unsigned long long fx = __ldcg(accfx + j);
+                const float sum = (fx >> 63) ? __int_as_float(0x7fc00000)
+                                             : (float)((double)fx * (1.0 / (double)kFxScale));
                 int lo = 0, hi = n_valid_probes;
                 while (lo < hi) {
                     const int mid = (lo + hi) >> 1;

@@ -561,6 +561,25 @@ def test_empty_selection_zeroes_the_output_and_the_cache_length(zipvl, name):
     assert n.item() == 0 and n2.item() == 0
 
 
+def test_a_nan_key_row_reaches_the_scores_and_is_reported_by_the_selection(zipvl):
+    """A NaN in one key row: the tensor-core score kernel (whose heads add their column sums into
+    fixed-point totals with integer atomics) still hands out NaN for that key's scores, and the
+    selection reports the bad value."""
+    layer = W.heavy_key_layer(L_visual=700, L_text=64, H=4, seed=33)
+    q, k, probe = layer.q.to(DEV), layer.k.clone(), layer.probe_pos.to(DEV)
+    k[300, 1, 5] = float("nan")
+    k = k.to(DEV)
+    desc = zipvl.layer_desc(q, k)
+    st = status_word()
+    acc, norm = zipvl.zipvl_score(desc, q, k, probe, status=st)
+    torch.cuda.synchronize()
+    assert torch.isnan(acc[300]).item() and torch.isnan(norm[300]).item()
+    st.zero_()
+    zipvl.zipvl_select(acc, norm, 0.9, status=st)
+    torch.cuda.synchronize()
+    assert st.item() & zipvl.DEV_BAD_VALUE
+
+
 def test_select_reports_negative_and_nan_scores(zipvl):
     g = torch.Generator().manual_seed(3)
     acc = torch.rand(500, generator=g).to(DEV)
