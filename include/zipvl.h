@@ -118,7 +118,8 @@ size_t zipvl_workspace_bytes(int32_t op, const zipvl_layer *layer, int32_t n_pro
  * random) is the caller's choice.  Entries outside [0,L) are skipped and
  * reported as ZIPVL_DEV_BAD_INDEX.  acc, norm: device float[L], written.
  * total: device double[1] or NULL.  ws: zipvl_workspace_bytes(ZIPVL_OP_SCORE).
- * The attention matrix A never reaches global memory.
+ * The attention matrix A never reaches global memory.  Two calls on the same inputs give the
+ * same bits (no floating-point sum depends on the order in which thread blocks finish).
  */
 zipvl_status zipvl_score(const zipvl_layer *layer, const void *q, const void *k,
                          const int32_t *probe_pos, int32_t n_probe, float *acc, float *norm,
