@@ -295,18 +295,40 @@ score_tc_kernel(const __grid_constant__ CUtensorMap kmap, LayerArgs a,
                 // probes below the warp's first key see none of its keys: whole 32-probe chunks of
                 // them are left out (probes ascend, the warp's rows too: lane 0 has the smallest bound)
                 const int first_vis_warp = __shfl_sync(0xffffffffu, first_vis, 0);
-                float cs4[4] = {0.f, 0.f, 0.f, 0.f};
+                // ... and from the last lane's bound on every probe sees all of the warp's keys: no
+                // test per element there.  Two elements per arithmetic instruction (packed fp32x2).
+                const int all_vis_warp = __shfl_sync(0xffffffffu, first_vis, 31);
+                const uint64_t scale2 = pack2f(a.scale_log2, a.scale_log2);
+                const uint64_t *nm2 = reinterpret_cast<const uint64_t *>(sNegM);
+                const uint64_t *il2 = reinterpret_cast<const uint64_t *>(sIl);
+                uint64_t cs2[4] = {0ull, 0ull, 0ull, 0ull};
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
                     if ((c + 1) * 32 <= first_vis_warp) continue;
+                    if (c * 32 >= all_vis_warp) {
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) {
-                        const int pr = c * 32 + e;
-                        // probes ascend, so "sees this key" is a prefix test on pr
-                        const float p = ex2(fmaf(__uint_as_float(sr[c][e]), a.scale_log2, sNegM[pr])) * sIl[pr];
-                        cs4[e & 3] += (pr >= first_vis) ? p : 0.f;
+                        for (int e = 0; e < 32; e += 2) {
+                            const int pr = c * 32 + e;
+                            float x0, x1;
+                            unpack2f(fma2(pack2u(sr[c][e], sr[c][e + 1]), scale2, nm2[pr >> 1]), x0, x1);
+                            cs2[(e >> 1) & 3] = fma2(pack2f(ex2(x0), ex2(x1)), il2[pr >> 1], cs2[(e >> 1) & 3]);
+                        }
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 32; e += 2) {
+                            const int pr = c * 32 + e;
+                            // probes ascend, so "sees this key" is a prefix test on pr
+                            float x0, x1;
+                            unpack2f(fma2(pack2u(sr[c][e], sr[c][e + 1]), scale2, nm2[pr >> 1]), x0, x1);
+                            const float p0 = (pr >= first_vis) ? ex2(x0) : 0.f;
+                            const float p1 = (pr + 1 >= first_vis) ? ex2(x1) : 0.f;
+                            cs2[(e >> 1) & 3] = fma2(pack2f(p0, p1), il2[pr >> 1], cs2[(e >> 1) & 3]);
+                        }
                     }
                 }
+                float cs4[4];
+                unpack2f(add2(cs2[0], cs2[1]), cs4[0], cs4[1]);
+                unpack2f(add2(cs2[2], cs2[3]), cs4[2], cs4[3]);
                 // the head's column sum goes into the column's fixed-point total (2^-40 units: a sum
                 // of 128 probabilities per head stays far below 2^63): integer adds commute, so the
                 // total does not depend on the order in which the heads arrive
